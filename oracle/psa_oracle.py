@@ -1,0 +1,287 @@
+"""CPU oracle for prefix-shared attention and the per-response log-prob gather.
+
+TEST INFRASTRUCTURE ONLY.  Nothing on the product path may import this module;
+it is used by the tests, by the smoke check and by the benchmark's CPU-baseline
+leg.  It shares no code with the CUDA library and imports nothing from the
+package.
+
+Everything is the plain textbook definition in float64 with an explicit dense
+boolean mask: no tiling, no online softmax, no block map.  A BLAS matmul is the
+only library primitive used as a step.
+
+Paper passages each function follows:
+
+* ``token_metadata`` / ``prefix_sharing_mask_packed``: Algorithm 3 ("Prefix
+  Sharing Mask with Packing"): causal AND same-document AND NOT(rejected query
+  looking at a chosen key), with dense per-token arrays I_chosen, I_rejected
+  and document ids D (Section 3.2).
+* ``prefix_sharing_mask_single``: Algorithm 1 ("Prefix Sharing Mask").
+* ``paired_packing_mask``: Algorithm 2 ("Attention Mask for Packing w/o Prefix
+  Sharing"): causal AND same per-token response id.
+* ``attention_fwd`` / ``attention_bwd``: Section 3.1: the attention computed
+  under the mask is ordinary softmax attention; the backward is its exact
+  gradient.
+* ``dpo_logp`` / ``paired_response_logps``: Section 2.1: the total log
+  probability of each completion given the prompt, recovered per response
+  from the packed row with the response boundaries (Section 3.2).
+* ``ideal_token_speedup`` / ``ideal_attention_speedup``: the two footnotes of
+  Section 4.2 (2(p+c)/(p+2c) and 2(p+c)^2/(2(p+c)^2-p^2)).
+
+Parity pins (tests/test_oracle_*.py): the paired-format equivalence claimed in
+Section 3.1 checked against torch's own scaled_dot_product_attention and
+autograd in float64, hand-derived mask fixtures, closed forms for q = 0,
+finite differences, torch.log_softmax for the gather.  No function here is
+"parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------
+# Masks
+# --------------------------------------------------------------------------
+
+def token_metadata(cu_seqlens, prefix_len, chosen_len, rejected_len):
+    """Dense per-token arrays of Algorithm 3 for one packed row (B = 1, L = T).
+
+    Returns (D, I_chosen, I_rejected), each int64 [T]: the document id of the
+    token's sample and the absolute start index, in the packed row, of that
+    sample's chosen and rejected completions.
+    """
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    n = len(cu) - 1
+    T = int(cu[n])
+    D = np.empty(T, dtype=np.int64)
+    Ic = np.empty(T, dtype=np.int64)
+    Ir = np.empty(T, dtype=np.int64)
+    for s in range(n):
+        P, C, R = int(prefix_len[s]), int(chosen_len[s]), int(rejected_len[s])
+        lo, hi = int(cu[s]), int(cu[s + 1])
+        if hi - lo != P + C + R:
+            raise ValueError("sample %d: cu_seqlens span %d != P+C+R = %d" % (s, hi - lo, P + C + R))
+        D[lo:hi] = s
+        Ic[lo:hi] = lo + P
+        Ir[lo:hi] = lo + P + C
+    return D, Ic, Ir
+
+
+def prefix_sharing_mask_packed(D, I_chosen, I_rejected):
+    """Algorithm 3, evaluated for every (q, kv) pair of the packed row.
+
+    mask[q, kv] = (kv <= q) and (D[q] == D[kv])
+                  and not ((I_rejected[q] <= q) and (I_chosen[q] <= kv < I_rejected[q]))
+    """
+    T = len(D)
+    q = np.arange(T, dtype=np.int64)[:, None]
+    kv = np.arange(T, dtype=np.int64)[None, :]
+    causal_mask = kv <= q
+    document_mask = D[:, None] == D[None, :]
+    chosen_ind = I_chosen[:, None]
+    rejected_ind = I_rejected[:, None]
+    dpo_mask = ~((rejected_ind <= q) & (chosen_ind <= kv) & (kv < rejected_ind))
+    return causal_mask & document_mask & dpo_mask
+
+
+def prefix_sharing_mask_single(L, chosen_ind, rejected_ind):
+    """Algorithm 1 for one unpacked sample of length L (scalar start indices)."""
+    q = np.arange(L, dtype=np.int64)[:, None]
+    kv = np.arange(L, dtype=np.int64)[None, :]
+    causal_mask = kv <= q
+    dpo_mask = ~((rejected_ind <= q) & (chosen_ind <= kv) & (kv < rejected_ind))
+    return causal_mask & dpo_mask
+
+
+def paired_packing_mask(response_ids):
+    """Algorithm 2: causal AND equal per-token response ids (paired layout)."""
+    Rid = np.asarray(response_ids, dtype=np.int64)
+    T = len(Rid)
+    q = np.arange(T, dtype=np.int64)[:, None]
+    kv = np.arange(T, dtype=np.int64)[None, :]
+    return (kv <= q) & (Rid[:, None] == Rid[None, :])
+
+
+def packed_mask(cu_seqlens, prefix_len, chosen_len, rejected_len):
+    """Convenience: Algorithm 3's mask straight from the per-sample lengths."""
+    return prefix_sharing_mask_packed(*token_metadata(cu_seqlens, prefix_len, chosen_len, rejected_len))
+
+
+def useful_pairs(prefix_len, chosen_len, rejected_len):
+    """Number of unmasked (q, kv) pairs per head, counted from the lengths:
+    the causal triangle over prompt+chosen, plus for the rejected rows the
+    prompt rectangle and their own causal triangle."""
+    U = 0
+    for P, C, R in zip(prefix_len, chosen_len, rejected_len):
+        P, C, R = int(P), int(C), int(R)
+        U += (P + C) * (P + C + 1) // 2 + R * P + R * (R + 1) // 2
+    return U
+
+
+def ideal_token_speedup(p, c):
+    """Footnote of Section 4.2.1: paired tokens / shared tokens = 2(p+c)/(p+2c)."""
+    return 2.0 * (p + c) / (p + 2.0 * c)
+
+
+def ideal_attention_speedup(p, c):
+    """Footnote of Section 4.2.2: 2(p+c)^2 / (2(p+c)^2 - p^2)."""
+    return 2.0 * (p + c) ** 2 / (2.0 * (p + c) ** 2 - p ** 2)
+
+
+# --------------------------------------------------------------------------
+# Attention, forward and backward, dense mask, float64
+# --------------------------------------------------------------------------
+
+def _as_f64(x):
+    return np.ascontiguousarray(np.asarray(x, dtype=np.float64))
+
+
+def attention_fwd(q, k, v, mask, softmax_scale=None):
+    """Masked softmax attention.
+
+    q [T, Hq, d]; k, v [T, Hkv, d]; mask bool [T, T] (True = may attend).
+    Query head h reads kv head h // (Hq // Hkv).
+    Returns o [T, Hq, d] and lse [Hq, T] = log sum_j exp(scale * q_i . k_j)
+    over the allowed j (natural log).  Every row must allow at least one key.
+    """
+    q, k, v = _as_f64(q), _as_f64(k), _as_f64(v)
+    T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    g = Hq // Hkv
+    scale = (1.0 / np.sqrt(d)) if softmax_scale is None else float(softmax_scale)
+    o = np.empty((T, Hq, d), dtype=np.float64)
+    lse = np.empty((Hq, T), dtype=np.float64)
+    for h in range(Hq):
+        kh = k[:, h // g, :]
+        vh = v[:, h // g, :]
+        S = scale * (q[:, h, :] @ kh.T)
+        S = np.where(mask, S, -np.inf)
+        m = S.max(axis=1)
+        E = np.exp(S - m[:, None])
+        l = E.sum(axis=1)
+        lse[h] = m + np.log(l)
+        P = E / l[:, None]
+        o[:, h, :] = P @ vh
+    return o, lse
+
+
+def attention_bwd(q, k, v, d_o, mask, softmax_scale=None):
+    """Exact gradient of attention_fwd for the loss sum(o * d_o).
+
+    Returns dq [T, Hq, d], dk, dv [T, Hkv, d]; dk, dv are summed over the
+    query heads that share a kv head.
+        P   = softmax(S) on the allowed pairs
+        dV  = P^T dO           dP = dO V^T
+        D_i = dO_i . o_i       dS = P * (dP - D)
+        dQ  = scale * dS K     dK = scale * dS^T Q
+    """
+    q, k, v, d_o = _as_f64(q), _as_f64(k), _as_f64(v), _as_f64(d_o)
+    T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    g = Hq // Hkv
+    scale = (1.0 / np.sqrt(d)) if softmax_scale is None else float(softmax_scale)
+    dq = np.zeros((T, Hq, d), dtype=np.float64)
+    dk = np.zeros((T, Hkv, d), dtype=np.float64)
+    dv = np.zeros((T, Hkv, d), dtype=np.float64)
+    for h in range(Hq):
+        kh = k[:, h // g, :]
+        vh = v[:, h // g, :]
+        qh = q[:, h, :]
+        doh = d_o[:, h, :]
+        S = scale * (qh @ kh.T)
+        S = np.where(mask, S, -np.inf)
+        m = S.max(axis=1)
+        E = np.exp(S - m[:, None])
+        P = E / E.sum(axis=1)[:, None]
+        oh = P @ vh
+        Dvec = (doh * oh).sum(axis=1)
+        dP = doh @ vh.T
+        dS = P * (dP - Dvec[:, None])
+        dq[:, h, :] = scale * (dS @ kh)
+        dk[:, h // g, :] += scale * (dS.T @ qh)
+        dv[:, h // g, :] += P.T @ doh
+    return dq, dk, dv
+
+
+def attention_rows(q, k, v, mask_rows, rows, softmax_scale=None):
+    """attention_fwd restricted to the query rows `rows` (for sampled checks at
+    sizes where the full T x T problem is too slow).  mask_rows is the
+    corresponding [len(rows), T] slice of the dense mask."""
+    q, k, v = _as_f64(q), _as_f64(k), _as_f64(v)
+    T, Hq, d = q.shape
+    g = Hq // k.shape[1]
+    scale = (1.0 / np.sqrt(d)) if softmax_scale is None else float(softmax_scale)
+    rows = np.asarray(rows, dtype=np.int64)
+    o = np.empty((len(rows), Hq, d), dtype=np.float64)
+    lse = np.empty((Hq, len(rows)), dtype=np.float64)
+    for h in range(Hq):
+        S = scale * (q[rows, h, :] @ k[:, h // g, :].T)
+        S = np.where(mask_rows, S, -np.inf)
+        m = S.max(axis=1)
+        E = np.exp(S - m[:, None])
+        l = E.sum(axis=1)
+        lse[h] = m + np.log(l)
+        o[:, h, :] = (E / l[:, None]) @ v[:, h // g, :]
+    return o, lse
+
+
+# --------------------------------------------------------------------------
+# Per-response summed log-probabilities
+# --------------------------------------------------------------------------
+
+def row_logprob(logits_row, target):
+    """log softmax(logits_row)[target] in float64."""
+    x = np.asarray(logits_row, dtype=np.float64)
+    m = x.max()
+    return float(x[int(target)] - (m + np.log(np.exp(x - m).sum())))
+
+
+def dpo_logp(logits, targets, segment_ids, n_segments,
+             fork_rows=(), fork_targets=(), fork_segments=()):
+    """out[g] = sum of log softmax(logits[t])[y] over every scored (t, y) whose
+    response id is g.
+
+    Row t scores targets[t] for response segment_ids[t] (skipped when the id is
+    negative).  The fork list adds second labels: row fork_rows[f] also scores
+    fork_targets[f] for response fork_segments[f].  In the shared layout this
+    is the last prompt row, whose next token is both the first chosen and the
+    first rejected token.
+    """
+    logits = np.asarray(logits, dtype=np.float64)
+    out = np.zeros(int(n_segments), dtype=np.float64)
+    for t in range(logits.shape[0]):
+        g = int(segment_ids[t])
+        if g >= 0:
+            out[g] += row_logprob(logits[t], targets[t])
+    for r, y, g in zip(fork_rows, fork_targets, fork_segments):
+        if int(g) >= 0:
+            out[int(g)] += row_logprob(logits[int(r)], y)
+    return out
+
+
+def paired_response_logps(logits_fn, token_ids, cu_seqlens, prefix_len, chosen_len, rejected_len):
+    """The paired-format definition of Section 2.1, written out.
+
+    For every sample build the two ordinary sequences [prompt | chosen] and
+    [prompt | rejected]; position i of a sequence predicts token i+1; the
+    response's log-prob is the sum over its own tokens.  `logits_fn(rows)`
+    returns the logits of the given packed-row indices (so that a paired
+    sequence can be assembled by copying rows of the shared layout).
+    Returns float64 [2n]: entry 2s = chosen, 2s+1 = rejected.
+    """
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    tok = np.asarray(token_ids, dtype=np.int64)
+    n = len(cu) - 1
+    out = np.zeros(2 * n, dtype=np.float64)
+    for s in range(n):
+        P, C, R = int(prefix_len[s]), int(chosen_len[s]), int(rejected_len[s])
+        ds = int(cu[s])
+        prompt = np.arange(ds, ds + P)
+        for which, resp in ((0, np.arange(ds + P, ds + P + C)),
+                            (1, np.arange(ds + P + C, ds + P + C + R))):
+            seq = np.concatenate([prompt, resp])
+            lg = np.asarray(logits_fn(seq), dtype=np.float64)
+            for i in range(len(seq) - 1):
+                nxt = i + 1
+                if nxt >= P:
+                    out[2 * s + which] += row_logprob(lg[i], tok[seq[nxt]])
+    return out
