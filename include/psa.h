@@ -1,0 +1,191 @@
+/*
+ * psa.h -- C ABI of libpsa: prefix-shared attention (forward + backward) and the
+ * per-response log-prob gather for DPO training, for NVIDIA B200 (sm_100a).
+ *
+ * Method: "Accelerating Direct Preference Optimization with Prefix Sharing"
+ * (arXiv 2410.20305).  Each training sample is ONE sequence
+ * [prompt | chosen | rejected]; samples are packed back to back into one row of
+ * T tokens.  A query may attend to a key iff (Algorithm 3, "Prefix Sharing Mask
+ * with Packing"):
+ *     key index <= query index                       (causal)
+ *     and both tokens belong to the same sample      (document mask)
+ *     and not (query is a rejected token and key is a chosen token).
+ * Algorithm 1 is the one-sample case; Algorithm 2 (the paired baseline layout)
+ * is the case rejected_len = 0 with 2n samples.
+ *
+ * Conventions
+ *   - Every function returns a psa_status_t and throws nothing.
+ *   - "host" pointers are ordinary CPU memory; "device" pointers are CUDA global
+ *     memory of the current device.  The library never takes ownership of a
+ *     caller's buffer and never allocates tensors; it allocates only the small
+ *     metadata owned by a plan.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Kernel launches are asynchronous on that stream.
+ *   - Tensor layout is token-major: element (t, h, c) of a [T, H, d] tensor is at
+ *     index (t*H + h)*d + c; bf16 storage.  lse is [Hq, T] float32.
+ *   - Query head h reads kv head h / (Hq / Hkv)  (grouped-query attention).
+ *   - Device base pointers must be 16-byte aligned (tiles are moved by TMA).
+ */
+#ifndef PSA_H_
+#define PSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct psa_plan psa_plan_t; /* opaque */
+
+typedef enum {
+  PSA_OK = 0,
+  PSA_ERR_INVALID_ARG = 1,          /* null pointer, negative size, bad enum, plan without device copy */
+  PSA_ERR_INCONSISTENT_LENGTHS = 2, /* cu_seqlens does not match prefix+chosen+rejected */
+  PSA_ERR_UNSUPPORTED = 3,          /* head_dim not in {64,128}, Hq % Hkv != 0, size over a stated maximum */
+  PSA_ERR_ALIGNMENT = 4,            /* a device pointer is not 16-byte aligned */
+  PSA_ERR_CUDA = 5,                 /* a CUDA runtime / driver call failed (no device, launch error, ...) */
+  PSA_ERR_DEVICE_STATUS = 6,        /* reserved: a kernel reported bad data through a status word */
+  PSA_ERR_TIMEOUT = 7               /* reserved: a bounded device-side wait expired */
+} psa_status_t;
+
+/* Bits of the word a kernel ORs into `device_status` (device int32, may be NULL). */
+#define PSA_DEVSTAT_WAIT_EXPIRED 1 /* a bounded barrier wait gave up; outputs are invalid    */
+#define PSA_DEVSTAT_BAD_TARGET   2 /* dpo_logp: a scored target id was outside [0, vocab)    */
+#define PSA_DEVSTAT_BAD_SEGMENT  4 /* dpo_logp: a segment id was >= n_segments               */
+
+/* Flags of psa_plan(). */
+#define PSA_PLAN_HOST_ONLY 1 /* build the tile map on the host only; no CUDA call is made */
+
+const char* psa_status_string(psa_status_t s);
+
+/*
+ * psa_plan -- build the block-sparsity tile map of the Algorithm 3 mask once per
+ * training step (Section 3.1: the sparse block mask is computed at the start of
+ * every step and handed to every attention layer; fully masked blocks are
+ * skipped).  One plan serves every layer and both psa_fwd and psa_bwd.
+ *
+ *   cu_seqlens   host int32 [n_samples+1]: first packed-row index of each sample,
+ *                cu_seqlens[0] = 0, cu_seqlens[n] = T.
+ *   prefix_len, chosen_len, rejected_len
+ *                host int32 [n_samples]: P, C, R >= 0 per sample, with
+ *                cu_seqlens[s+1] - cu_seqlens[s] = P + C + R.  Any of them may
+ *                be 0 (R = 0 is plain packed causal attention).
+ *   n_q_heads, n_kv_heads, head_dim
+ *                Hq % Hkv == 0; head_dim 64 or 128.
+ *   softmax_scale  multiplies q.k before the softmax; <= 0 selects 1/sqrt(head_dim).
+ *   flags        0 or PSA_PLAN_HOST_ONLY.
+ *   stream       the upload of the tile map is enqueued here (ignored if HOST_ONLY).
+ *   out          receives the plan; destroy with psa_plan_destroy.
+ *
+ * Tiles are 128 x 128 and aligned to the start of each sample.  A (query tile,
+ * key tile) pair is dropped when every pair in it is masked, marked FULL when
+ * none is, and PARTIAL otherwise (masked per element in registers).
+ * Errors: INVALID_ARG, INCONSISTENT_LENGTHS, UNSUPPORTED, CUDA.
+ */
+psa_status_t psa_plan(const int32_t* cu_seqlens, const int32_t* prefix_len,
+                      const int32_t* chosen_len, const int32_t* rejected_len,
+                      int32_t n_samples, int32_t n_q_heads, int32_t n_kv_heads,
+                      int32_t head_dim, float softmax_scale, int32_t flags,
+                      void* stream, psa_plan_t** out);
+
+/* Copies a HOST_ONLY plan's tile map to the current device (no-op if already there). */
+psa_status_t psa_plan_upload(psa_plan_t* plan, void* stream);
+
+/* Frees the plan's host and device metadata.  NULL is accepted. */
+psa_status_t psa_plan_destroy(psa_plan_t* plan);
+
+/*
+ * psa_plan_stats -- any output pointer may be NULL.
+ *   total_tokens        T
+ *   useful_pairs        unmasked (q, kv) pairs per query head
+ *   live_tiles          (query tile, key tile) pairs kept in the map
+ *   partial_tiles       how many of those need per-element masking in the forward
+ *   bwd_workspace_bytes size of the device scratch buffer psa_bwd needs
+ */
+psa_status_t psa_plan_stats(const psa_plan_t* plan, int64_t* total_tokens,
+                            int64_t* useful_pairs, int64_t* live_tiles,
+                            int64_t* partial_tiles, size_t* bwd_workspace_bytes);
+
+/*
+ * psa_plan_counts / psa_plan_export -- read the tile map back (tests, tools).
+ * direction 0 = forward map (one record per query tile, entries = key tiles),
+ * direction 1 = transposed map for the backward (one record per key tile,
+ * entries = query tiles).
+ * A record is 8 int32: { row0, sample_start, local0, sample_len, chosen_start,
+ * rejected_start, entry_offset, entry_count }, where row0 is the packed-row
+ * index of the tile's first row, local0 = row0 - sample_start, and
+ * chosen_start / rejected_start are relative to sample_start.  An entry is
+ * (tile_index_within_sample << 1) | needs_mask.
+ * `tiles` is host int32 [n_tiles*8], `entries` host int32 [n_entries].
+ */
+psa_status_t psa_plan_counts(const psa_plan_t* plan, int32_t direction,
+                             int32_t* n_tiles, int32_t* n_entries);
+psa_status_t psa_plan_export(const psa_plan_t* plan, int32_t direction,
+                             int32_t* tiles, int32_t* entries);
+
+/*
+ * psa_fwd -- attention forward under the plan's mask (Section 3.1).
+ *   S = scale * Q K^T on the live tiles, softmax over the allowed keys of each
+ *   row in fp32, O = P V;  lse[h][t] = log sum_j exp(S[t][j])  (natural log).
+ *   q        device bf16 [T, Hq, d]        k, v   device bf16 [T, Hkv, d]
+ *   o        device bf16 [T, Hq, d] (out)  lse    device fp32 [Hq, T] (out)
+ *   device_status  device int32 or NULL; bits are ORed in, never cleared.
+ * Rows >= T are neither read nor written.  T = 0 is a no-op.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA.
+ */
+psa_status_t psa_fwd(const psa_plan_t* plan, const void* q, const void* k, const void* v,
+                     void* o, float* lse, int32_t* device_status, void* stream);
+
+/*
+ * psa_bwd -- exact gradient of psa_fwd; probabilities are recomputed from lse.
+ *   D_i = dO_i . O_i;  P = exp(S - lse);  dV = P^T dO;  dP = dO V^T;
+ *   dS = P * (dP - D);  dQ = scale * dS K;  dK = scale * dS^T Q;
+ *   dK and dV are summed over the Hq/Hkv query heads of each kv head.
+ *   d_o, q, o   device bf16 [T, Hq, d]     k, v    device bf16 [T, Hkv, d]
+ *   lse         device fp32 [Hq, T] as written by psa_fwd
+ *   dq          device bf16 [T, Hq, d] (out)   dk, dv  device bf16 [T, Hkv, d] (out)
+ *   workspace   device scratch of psa_plan_stats().bwd_workspace_bytes bytes,
+ *               256-byte aligned; contents on entry are ignored, on exit undefined.
+ * The call is stateless: the same plan may serve any number of layers.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA.
+ */
+psa_status_t psa_bwd(const psa_plan_t* plan, const void* d_o, const void* q, const void* k,
+                     const void* v, const void* o, const float* lse,
+                     void* dq, void* dk, void* dv, void* workspace,
+                     int32_t* device_status, void* stream);
+
+/*
+ * dpo_logp -- summed log-probabilities per response (Section 2.1: the total
+ * log probability of each completion; Section 3.2: responses are recovered at
+ * loss time from their boundaries).
+ *   out[g] = sum over scored (row t, label y) with response id g of
+ *            logits[t][y] - log sum_v exp(logits[t][v])
+ *   logits        device [n_rows, vocab], row stride `row_stride` elements
+ *   logits_dtype  PSA_DTYPE_F32 or PSA_DTYPE_BF16
+ *   targets       device int32 [n_rows]: label scored by row t
+ *   segment_ids   device int32 [n_rows]: response id of that label, or < 0 if the
+ *                 row scores nothing through this array (its logits are then not
+ *                 read unless a fork names the row)
+ *   fork_rows, fork_targets, fork_segments
+ *                 device int32 [n_forks] (may be NULL when n_forks = 0): rows that
+ *                 score a SECOND label.  In the shared layout the last prompt row
+ *                 predicts both the first chosen and the first rejected token.
+ *   out           device fp32 [n_segments], overwritten
+ *   device_status device int32 or NULL: PSA_DEVSTAT_BAD_TARGET / BAD_SEGMENT are
+ *                 ORed in and the offending label is skipped; nothing faults.
+ * Accumulation is fp32; the order of the per-row additions into out[] is not fixed.
+ * Errors: INVALID_ARG, ALIGNMENT (rows must start 16-byte aligned), CUDA.
+ */
+#define PSA_DTYPE_F32 0
+#define PSA_DTYPE_BF16 1
+psa_status_t dpo_logp(const void* logits, int32_t logits_dtype, int64_t n_rows, int64_t vocab,
+                      int64_t row_stride, const int32_t* targets, const int32_t* segment_ids,
+                      const int32_t* fork_rows, const int32_t* fork_targets,
+                      const int32_t* fork_segments, int32_t n_forks, int32_t n_segments,
+                      float* out, int32_t* device_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSA_H_ */

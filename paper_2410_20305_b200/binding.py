@@ -1,0 +1,204 @@
+"""Thin ctypes binding of libpsa's C ABI (include/psa.h).
+
+Argument marshalling only: every step of the path runs inside the library's
+CUDA kernels.  torch is used for device memory and streams.  There is no CPU
+fallback: if the shared library is missing or a call fails, an exception is
+raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libpsa.so")
+_lib = None
+
+PSA_PLAN_HOST_ONLY = 1
+PSA_DTYPE_F32, PSA_DTYPE_BF16 = 0, 1
+PSA_DEVSTAT_WAIT_EXPIRED, PSA_DEVSTAT_BAD_TARGET, PSA_DEVSTAT_BAD_SEGMENT = 1, 2, 4
+
+EXPORTED_SYMBOLS = (
+    "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
+    "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp",
+)
+
+
+class PsaError(RuntimeError):
+    def __init__(self, fn, code, text):
+        super().__init__("%s failed: status %d (%s)" % (fn, code, text))
+        self.code = code
+
+
+def load_library():
+    """Loads libpsa.so (building it first if the sources are newer and nvcc is
+    present).  Raises if the library cannot be had."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    from . import build as _build
+    try:
+        _build.build()
+    except Exception:
+        if not os.path.exists(_LIB_PATH):
+            raise
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError("libpsa.so is missing and could not be built: %s" % _LIB_PATH)
+    lib = C.CDLL(_LIB_PATH)
+    vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+    lib.psa_status_string.restype = C.c_char_p
+    lib.psa_status_string.argtypes = [C.c_int]
+    lib.psa_plan.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, f32, i32, vp, C.POINTER(vp)]
+    lib.psa_plan_upload.argtypes = [vp, vp]
+    lib.psa_plan_destroy.argtypes = [vp]
+    lib.psa_plan_stats.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), C.POINTER(i64), C.POINTER(i64),
+                                   C.POINTER(C.c_size_t)]
+    lib.psa_plan_counts.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(i32)]
+    lib.psa_plan_export.argtypes = [vp, i32, vp, vp]
+    lib.psa_fwd.argtypes = [vp] * 8
+    lib.psa_bwd.argtypes = [vp] * 13
+    lib.dpo_logp.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
+    for name in EXPORTED_SYMBOLS:
+        if name != "psa_status_string":
+            getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _check(fn, code):
+    if code != 0:
+        raise PsaError(fn, code, load_library().psa_status_string(code).decode())
+
+
+def _i32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _stream(stream):
+    if stream is not None:
+        return C.c_void_p(int(stream))
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream) if torch.cuda.is_available() else C.c_void_p(0)
+
+
+def _ptr(t):
+    return C.c_void_p(0) if t is None else C.c_void_p(t.data_ptr())
+
+
+class Plan:
+    """Owner of a psa_plan_t*.  One plan serves every layer of a step."""
+
+    def __init__(self, handle, n_q_heads, n_kv_heads, head_dim):
+        self._h = handle
+        self.n_q_heads, self.n_kv_heads, self.head_dim = n_q_heads, n_kv_heads, head_dim
+        lib = load_library()
+        T, U, live, part = C.c_int64(), C.c_int64(), C.c_int64(), C.c_int64()
+        ws = C.c_size_t()
+        _check("psa_plan_stats", lib.psa_plan_stats(self._h, C.byref(T), C.byref(U), C.byref(live), C.byref(part),
+                                                    C.byref(ws)))
+        self.total_tokens, self.useful_pairs = T.value, U.value
+        self.live_tiles, self.partial_tiles, self.bwd_workspace_bytes = live.value, part.value, ws.value
+
+    def upload(self, stream=None):
+        _check("psa_plan_upload", load_library().psa_plan_upload(self._h, _stream(stream)))
+
+    def export(self, direction):
+        """Tile records int32 [n_tiles, 8] and entries int32 [n_entries] of the
+        forward (0) or transposed (1) map."""
+        lib = load_library()
+        nt, ne = C.c_int32(), C.c_int32()
+        _check("psa_plan_counts", lib.psa_plan_counts(self._h, direction, C.byref(nt), C.byref(ne)))
+        tiles = np.zeros((max(nt.value, 1), 8), dtype=np.int32)
+        entries = np.zeros(max(ne.value, 1), dtype=np.int32)
+        _check("psa_plan_export", lib.psa_plan_export(self._h, direction, tiles.ctypes.data, entries.ctypes.data))
+        return tiles[:nt.value], entries[:ne.value]
+
+    def close(self):
+        if self._h:
+            h, self._h = self._h, None
+            load_library().psa_plan_destroy(h)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def psa_plan(cu_seqlens, prefix_len, chosen_len, rejected_len, n_q_heads, n_kv_heads, head_dim,
+             softmax_scale=0.0, host_only=False, stream=None) -> Plan:
+    lib = load_library()
+    cu, P, Cc, R = _i32(cu_seqlens), _i32(prefix_len), _i32(chosen_len), _i32(rejected_len)
+    n = len(P)
+    if len(cu) != n + 1 or len(Cc) != n or len(R) != n:
+        raise ValueError("cu_seqlens must have n+1 entries and the three length arrays n entries")
+    out = C.c_void_p()
+    flags = PSA_PLAN_HOST_ONLY if host_only else 0
+    st = C.c_void_p(0) if host_only else _stream(stream)
+    _check("psa_plan", lib.psa_plan(cu.ctypes.data, P.ctypes.data, Cc.ctypes.data, R.ctypes.data, n, n_q_heads,
+                                    n_kv_heads, head_dim, float(softmax_scale), flags, st, C.byref(out)))
+    return Plan(out, n_q_heads, n_kv_heads, head_dim)
+
+
+def psa_fwd(plan: Plan, q, k, v, o=None, lse=None, status=None, stream=None):
+    """q [T,Hq,d], k, v [T,Hkv,d] bf16 CUDA tensors -> (o [T,Hq,d] bf16, lse [Hq,T] fp32)."""
+    import torch
+    T = plan.total_tokens
+    assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous() and tuple(q.shape) == (T, plan.n_q_heads, plan.head_dim)
+    for t in (k, v):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and tuple(t.shape) == (T, plan.n_kv_heads, plan.head_dim)
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((plan.n_q_heads, T), dtype=torch.float32, device=q.device)
+    _check("psa_fwd", load_library().psa_fwd(plan._h, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(status),
+                                             _stream(stream)))
+    return o, lse
+
+
+def psa_bwd(plan: Plan, d_o, q, k, v, o, lse, dq=None, dk=None, dv=None, workspace=None, status=None, stream=None):
+    """Returns (dq [T,Hq,d], dk, dv [T,Hkv,d]) bf16."""
+    import torch
+    for t in (d_o, q, k, v, o):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    assert lse.dtype == torch.float32 and lse.is_contiguous()
+    if dq is None:
+        dq = torch.empty_like(q)
+    if dk is None:
+        dk = torch.empty_like(k)
+    if dv is None:
+        dv = torch.empty_like(v)
+    if workspace is None:
+        workspace = torch.empty(max(plan.bwd_workspace_bytes, 256), dtype=torch.uint8, device=q.device)
+    assert workspace.numel() * workspace.element_size() >= plan.bwd_workspace_bytes
+    _check("psa_bwd", load_library().psa_bwd(plan._h, _ptr(d_o), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
+                                             _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace), _ptr(status),
+                                             _stream(stream)))
+    return dq, dk, dv
+
+
+def dpo_logp(logits, targets, segment_ids, n_segments, fork_rows=None, fork_targets=None, fork_segments=None,
+             out=None, status=None, stream=None):
+    """logits [n_rows, vocab] fp32 or bf16 (rows may be strided), targets / segment_ids
+    int32 [n_rows], optional fork arrays int32 [n_forks] -> out fp32 [n_segments]."""
+    import torch
+    assert logits.is_cuda and logits.dim() == 2 and logits.stride(1) == 1
+    dt = {torch.float32: PSA_DTYPE_F32, torch.bfloat16: PSA_DTYPE_BF16}[logits.dtype]
+    n_rows, vocab = logits.shape
+    for t in (targets, segment_ids):
+        assert t.is_cuda and t.dtype == torch.int32 and t.is_contiguous() and t.numel() == n_rows
+    n_forks = 0 if fork_rows is None else int(fork_rows.numel())
+    if n_forks:
+        for t in (fork_rows, fork_targets, fork_segments):
+            assert t.is_cuda and t.dtype == torch.int32 and t.is_contiguous() and t.numel() == n_forks
+    else:
+        fork_rows = fork_targets = fork_segments = None
+    if out is None:
+        out = torch.empty(n_segments, dtype=torch.float32, device=logits.device)
+    _check("dpo_logp", load_library().dpo_logp(_ptr(logits), dt, n_rows, vocab, logits.stride(0) if n_rows > 1 else vocab,
+                                               _ptr(targets), _ptr(segment_ids), _ptr(fork_rows), _ptr(fork_targets),
+                                               _ptr(fork_segments), n_forks, n_segments, _ptr(out), _ptr(status),
+                                               _stream(stream)))
+    return out

@@ -1,0 +1,58 @@
+// Internal definitions shared by the host planner and the kernel launchers.
+#pragma once
+#include <cstdint>
+#include <vector>
+
+#include "psa.h"
+
+namespace psa {
+
+constexpr int kTile = 128;  // query-tile and key-tile edge, in tokens
+
+// One record per query tile (forward map) or per key tile (transposed map).
+// All positions except row0 / ds are relative to the sample start.
+struct TileRec {
+  int32_t row0;      // packed-row index of the tile's first row
+  int32_t ds;        // packed-row index of the sample's first token
+  int32_t local0;    // row0 - ds
+  int32_t len;       // sample length P + C + R
+  int32_t cs;        // chosen start  = P
+  int32_t rs;        // rejected start = P + C
+  int32_t list_off;  // first entry of this tile's list
+  int32_t list_cnt;  // number of live partner tiles
+};
+static_assert(sizeof(TileRec) == 32, "TileRec is 8 int32");
+
+}  // namespace psa
+
+struct psa_plan {
+  int32_t n_samples = 0, T = 0, Hq = 0, Hkv = 0, d = 0;
+  float scale = 0.f;
+  int64_t useful_pairs = 0, live_tiles = 0, partial_tiles = 0;
+  size_t bwd_workspace_bytes = 0;
+  std::vector<psa::TileRec> q_tiles, kv_tiles;   // sorted, longest list first
+  std::vector<int32_t> fwd_entries, bwd_entries;
+  // device copy (one allocation)
+  int device = -1;
+  void* d_blob = nullptr;
+  const psa::TileRec* d_q_tiles = nullptr;
+  const psa::TileRec* d_kv_tiles = nullptr;
+  const int32_t* d_fwd_entries = nullptr;
+  const int32_t* d_bwd_entries = nullptr;
+};
+
+namespace psa {
+// Workspace layout of psa_bwd (byte offsets, each 256-aligned).
+struct BwdWorkspace {
+  size_t dq_accum_off, dq_accum_bytes;  // fp32 [T, Hq, d]
+  size_t delta_off, delta_bytes;        // fp32 [Hq, Tpad]  D_i = dO_i . O_i
+  size_t total;
+};
+BwdWorkspace bwd_workspace_layout(int64_t T, int Hq, int d);
+
+psa_status_t launch_fwd(const psa_plan_t* plan, const void* q, const void* k, const void* v, void* o,
+                        float* lse, int32_t* device_status, void* stream);
+psa_status_t launch_bwd(const psa_plan_t* plan, const void* d_o, const void* q, const void* k,
+                        const void* v, const void* o, const float* lse, void* dq, void* dk, void* dv,
+                        void* workspace, int32_t* device_status, void* stream);
+}  // namespace psa

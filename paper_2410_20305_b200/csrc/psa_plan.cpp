@@ -1,0 +1,221 @@
+// Host planner: block-sparsity tile map of the prefix-sharing mask with packing
+// (Algorithm 3), built once per step and reused by every layer (Section 3.1).
+//
+// Tiles are 128 x 128 and aligned to each sample's first token, so that within a
+// sample query tile i and key tile j cover local rows [128 i, 128 i + 128) and
+// [128 j, 128 j + 128).  In local coordinates (cs = P, rs = P + C, len = P+C+R)
+// the mask is:  kv <= q  and not (q >= rs and cs <= kv < rs).
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <numeric>
+
+#include "psa_internal.h"
+
+namespace psa {
+
+BwdWorkspace bwd_workspace_layout(int64_t T, int Hq, int d) {
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  BwdWorkspace w{};
+  int64_t Tpad = (T + kTile - 1) / kTile * kTile + kTile;
+  w.dq_accum_off = 0;
+  w.dq_accum_bytes = up(size_t(T) * Hq * d * sizeof(float));
+  w.delta_off = w.dq_accum_off + w.dq_accum_bytes;
+  w.delta_bytes = up(size_t(Hq) * Tpad * sizeof(float));
+  w.total = w.delta_off + w.delta_bytes;
+  return w;
+}
+
+namespace {
+
+// Classification of tile pair (i, j) of one sample.  Returns 0 = dropped,
+// 1 = live and full, 2 = live and needs masking.  `bwd` also requires the rows
+// past the sample's end (ragged last query tile) to be masked.
+int classify(int i, int j, int len, int cs, int rs, bool bwd) {
+  if (j > i) return 0;
+  const int q0 = i * kTile, q1 = std::min(q0 + kTile, len);  // valid query rows
+  const int k0 = j * kTile, k1 = std::min(k0 + kTile, len);  // valid key rows
+  if (j == i) return 2;  // the diagonal tile always holds the row's own key
+  // j < i: causality holds for every pair.  Forbidden rectangle: q >= rs, cs <= kv < rs.
+  const bool rows_all_rejected = q0 >= rs;
+  const bool rows_some_rejected = q1 > rs;        // q1 - 1 >= rs
+  const bool keys_all_chosen = k0 >= cs && k1 <= rs;
+  const bool keys_some_chosen = k1 > cs && k0 < rs;
+  if (rows_all_rejected && keys_all_chosen) return 0;
+  bool partial = rows_some_rejected && keys_some_chosen;
+  if (bwd && q0 + kTile > len) partial = true;
+  return partial ? 2 : 1;
+}
+
+}  // namespace
+}  // namespace psa
+
+using psa::kTile;
+using psa::TileRec;
+
+extern "C" const char* psa_status_string(psa_status_t s) {
+  switch (s) {
+    case PSA_OK: return "ok";
+    case PSA_ERR_INVALID_ARG: return "invalid argument";
+    case PSA_ERR_INCONSISTENT_LENGTHS: return "cu_seqlens inconsistent with prefix/chosen/rejected lengths";
+    case PSA_ERR_UNSUPPORTED: return "unsupported configuration";
+    case PSA_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+    case PSA_ERR_CUDA: return "CUDA call failed";
+    case PSA_ERR_DEVICE_STATUS: return "kernel reported bad data";
+    case PSA_ERR_TIMEOUT: return "bounded device wait expired";
+  }
+  return "unknown status";
+}
+
+extern "C" psa_status_t psa_plan(const int32_t* cu_seqlens, const int32_t* prefix_len,
+                                 const int32_t* chosen_len, const int32_t* rejected_len,
+                                 int32_t n_samples, int32_t n_q_heads, int32_t n_kv_heads,
+                                 int32_t head_dim, float softmax_scale, int32_t flags,
+                                 void* stream, psa_plan_t** out) {
+  if (!out) return PSA_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (n_samples < 0 || !cu_seqlens) return PSA_ERR_INVALID_ARG;
+  if (n_samples > 0 && (!prefix_len || !chosen_len || !rejected_len)) return PSA_ERR_INVALID_ARG;
+  if (n_q_heads <= 0 || n_kv_heads <= 0) return PSA_ERR_INVALID_ARG;
+  if (flags & ~PSA_PLAN_HOST_ONLY) return PSA_ERR_INVALID_ARG;
+  if (n_q_heads % n_kv_heads != 0) return PSA_ERR_UNSUPPORTED;
+  if (head_dim != 64 && head_dim != 128) return PSA_ERR_UNSUPPORTED;
+  if (cu_seqlens[0] != 0) return PSA_ERR_INCONSISTENT_LENGTHS;
+  for (int s = 0; s < n_samples; ++s) {
+    if (prefix_len[s] < 0 || chosen_len[s] < 0 || rejected_len[s] < 0) return PSA_ERR_INVALID_ARG;
+    int64_t tot = int64_t(prefix_len[s]) + chosen_len[s] + rejected_len[s];
+    if (int64_t(cu_seqlens[s + 1]) - cu_seqlens[s] != tot) return PSA_ERR_INCONSISTENT_LENGTHS;
+  }
+  // Row indices, and row*heads products used for grid sizes, stay in int32.
+  if (int64_t(cu_seqlens[n_samples]) > (int64_t(1) << 30)) return PSA_ERR_UNSUPPORTED;
+
+  psa_plan_t* p = new (std::nothrow) psa_plan_t;
+  if (!p) return PSA_ERR_INVALID_ARG;
+  p->n_samples = n_samples;
+  p->T = cu_seqlens[n_samples];
+  p->Hq = n_q_heads;
+  p->Hkv = n_kv_heads;
+  p->d = head_dim;
+  p->scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt(float(head_dim));
+
+  for (int s = 0; s < n_samples; ++s) {
+    const int P = prefix_len[s], C = chosen_len[s], R = rejected_len[s];
+    const int len = P + C + R, cs = P, rs = P + C, ds = cu_seqlens[s];
+    p->useful_pairs += int64_t(P + C) * (P + C + 1) / 2 + int64_t(R) * P + int64_t(R) * (R + 1) / 2;
+    const int nt = (len + kTile - 1) / kTile;
+    for (int i = 0; i < nt; ++i) {  // forward: query tile i, its key tiles in ascending order
+      TileRec r{ds + i * kTile, ds, i * kTile, len, cs, rs, int32_t(p->fwd_entries.size()), 0};
+      for (int j = 0; j <= i; ++j) {
+        int c = psa::classify(i, j, len, cs, rs, false);
+        if (!c) continue;
+        p->fwd_entries.push_back((j << 1) | (c == 2));
+        ++r.list_cnt;
+        ++p->live_tiles;
+        p->partial_tiles += (c == 2);
+      }
+      p->q_tiles.push_back(r);
+    }
+    for (int j = 0; j < nt; ++j) {  // transposed: key tile j, its query tiles in ascending order
+      TileRec r{ds + j * kTile, ds, j * kTile, len, cs, rs, int32_t(p->bwd_entries.size()), 0};
+      for (int i = j; i < nt; ++i) {
+        int c = psa::classify(i, j, len, cs, rs, true);
+        if (!c) continue;
+        p->bwd_entries.push_back((i << 1) | (c == 2));
+        ++r.list_cnt;
+      }
+      p->kv_tiles.push_back(r);
+    }
+  }
+  // Longest list first: the hardware hands out CTAs in index order, so the long
+  // work items start early and the short ones fill the tail.
+  auto longest_first = [](const TileRec& a, const TileRec& b) { return a.list_cnt > b.list_cnt; };
+  std::stable_sort(p->q_tiles.begin(), p->q_tiles.end(), longest_first);
+  std::stable_sort(p->kv_tiles.begin(), p->kv_tiles.end(), longest_first);
+  p->bwd_workspace_bytes = psa::bwd_workspace_layout(p->T, p->Hq, p->d).total;
+
+  if (!(flags & PSA_PLAN_HOST_ONLY)) {
+    psa_status_t st = psa_plan_upload(p, stream);
+    if (st != PSA_OK) {
+      delete p;
+      return st;
+    }
+  }
+  *out = p;
+  return PSA_OK;
+}
+
+extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
+  if (!p) return PSA_ERR_INVALID_ARG;
+  if (p->d_blob) return PSA_OK;
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  const size_t b0 = up(p->q_tiles.size() * sizeof(TileRec));
+  const size_t b1 = up(p->kv_tiles.size() * sizeof(TileRec));
+  const size_t b2 = up(p->fwd_entries.size() * sizeof(int32_t));
+  const size_t b3 = up(p->bwd_entries.size() * sizeof(int32_t));
+  const size_t total = b0 + b1 + b2 + b3 + 256;
+  if (cudaGetDevice(&p->device) != cudaSuccess) return PSA_ERR_CUDA;
+  void* blob = nullptr;
+  if (cudaMalloc(&blob, total) != cudaSuccess) return PSA_ERR_CUDA;
+  // Stage in one host buffer so a single copy suffices; the copy is synchronous
+  // with respect to the host buffer because it is pageable memory.
+  std::vector<char> host(total, 0);
+  std::memcpy(host.data(), p->q_tiles.data(), p->q_tiles.size() * sizeof(TileRec));
+  std::memcpy(host.data() + b0, p->kv_tiles.data(), p->kv_tiles.size() * sizeof(TileRec));
+  std::memcpy(host.data() + b0 + b1, p->fwd_entries.data(), p->fwd_entries.size() * sizeof(int32_t));
+  std::memcpy(host.data() + b0 + b1 + b2, p->bwd_entries.data(), p->bwd_entries.size() * sizeof(int32_t));
+  if (cudaMemcpyAsync(blob, host.data(), total, cudaMemcpyHostToDevice, cudaStream_t(stream)) != cudaSuccess ||
+      cudaStreamSynchronize(cudaStream_t(stream)) != cudaSuccess) {
+    cudaFree(blob);
+    return PSA_ERR_CUDA;
+  }
+  char* b = static_cast<char*>(blob);
+  p->d_blob = blob;
+  p->d_q_tiles = reinterpret_cast<const TileRec*>(b);
+  p->d_kv_tiles = reinterpret_cast<const TileRec*>(b + b0);
+  p->d_fwd_entries = reinterpret_cast<const int32_t*>(b + b0 + b1);
+  p->d_bwd_entries = reinterpret_cast<const int32_t*>(b + b0 + b1 + b2);
+  return PSA_OK;
+}
+
+extern "C" psa_status_t psa_plan_destroy(psa_plan_t* p) {
+  if (!p) return PSA_OK;
+  psa_status_t st = PSA_OK;
+  if (p->d_blob && cudaFree(p->d_blob) != cudaSuccess) st = PSA_ERR_CUDA;
+  delete p;
+  return st;
+}
+
+extern "C" psa_status_t psa_plan_stats(const psa_plan_t* p, int64_t* total_tokens, int64_t* useful_pairs,
+                                       int64_t* live_tiles, int64_t* partial_tiles,
+                                       size_t* bwd_workspace_bytes) {
+  if (!p) return PSA_ERR_INVALID_ARG;
+  if (total_tokens) *total_tokens = p->T;
+  if (useful_pairs) *useful_pairs = p->useful_pairs;
+  if (live_tiles) *live_tiles = p->live_tiles;
+  if (partial_tiles) *partial_tiles = p->partial_tiles;
+  if (bwd_workspace_bytes) *bwd_workspace_bytes = p->bwd_workspace_bytes;
+  return PSA_OK;
+}
+
+extern "C" psa_status_t psa_plan_counts(const psa_plan_t* p, int32_t direction, int32_t* n_tiles,
+                                        int32_t* n_entries) {
+  if (!p || (direction != 0 && direction != 1)) return PSA_ERR_INVALID_ARG;
+  const auto& tiles = direction ? p->kv_tiles : p->q_tiles;
+  const auto& entries = direction ? p->bwd_entries : p->fwd_entries;
+  if (n_tiles) *n_tiles = int32_t(tiles.size());
+  if (n_entries) *n_entries = int32_t(entries.size());
+  return PSA_OK;
+}
+
+extern "C" psa_status_t psa_plan_export(const psa_plan_t* p, int32_t direction, int32_t* tiles,
+                                        int32_t* entries) {
+  if (!p || (direction != 0 && direction != 1) || !tiles || !entries) return PSA_ERR_INVALID_ARG;
+  const auto& t = direction ? p->kv_tiles : p->q_tiles;
+  const auto& e = direction ? p->bwd_entries : p->fwd_entries;
+  if (!t.empty()) std::memcpy(tiles, t.data(), t.size() * sizeof(TileRec));
+  if (!e.empty()) std::memcpy(entries, e.data(), e.size() * sizeof(int32_t));
+  return PSA_OK;
+}

@@ -1,0 +1,79 @@
+"""psa_fwd on the GPU against the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2410_20305_b200 import binding as B
+from paper_2410_20305_b200 import workloads as wl
+
+from gpu_util import TOL_LSE, TOL_O, device_plan, max_abs, oracle_fwd, read_status
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_fwd(pack, seed, scale=0.0, std=1.0):
+    q, k, v, _ = wl.attention_inputs(pack, seed, std=std)
+    plan = device_plan(pack, scale)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    T = pack.total_tokens
+    # canary rows after the outputs: the kernel must not write past T
+    o = torch.full((T + 4, pack.n_q_heads, pack.head_dim), 7.0, dtype=torch.bfloat16, device="cuda")
+    o_out, lse = B.psa_fwd(plan, q.cuda(), k.cuda(), v.cuda(), o=o[:T], status=status)
+    assert read_status(status) == 0
+    assert (o[T:] == 7.0).all()
+    ro, rl = oracle_fwd(pack, q, k, v, None if scale == 0.0 else scale)
+    return max_abs(o_out, ro), max_abs(lse, rl)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_tiny_config(seed):
+    eo, el = _run_fwd(wl.config_pack(0), seed)
+    assert eo <= TOL_O and el <= TOL_LSE, (eo, el)
+
+
+@pytest.mark.parametrize("d,hq,hkv", [(128, 4, 1), (128, 8, 8), (64, 8, 2), (64, 1, 1)])
+def test_random_ragged_packs(d, hq, hkv):
+    for seed in range(3):
+        pack = wl.random_pack(40 + seed, 4, 330, hq, hkv, d)
+        eo, el = _run_fwd(pack, seed)
+        assert eo <= TOL_O and el <= TOL_LSE, (seed, eo, el)
+
+
+def test_degenerate_lengths():
+    lengths = [(0, 70, 200), (300, 0, 45), (129, 255, 0), (1, 0, 0), (1, 1, 1), (128, 128, 128), (0, 0, 5)]
+    eo, el = _run_fwd(wl.pack_from_lengths("deg", lengths, 4, 2, 128), 5)
+    assert eo <= TOL_O and el <= TOL_LSE, (eo, el)
+
+
+def test_single_token_and_explicit_scale():
+    eo, el = _run_fwd(wl.pack_from_lengths("one", [(1, 0, 0)], 2, 2, 64), 1)
+    assert eo <= TOL_O and el <= TOL_LSE
+    eo, el = _run_fwd(wl.random_pack(77, 3, 200, 4, 4, 64), 2, scale=0.2)
+    assert eo <= TOL_O and el <= TOL_LSE, (eo, el)
+
+
+def test_long_sample_spans_many_tiles():
+    pack = wl.pack_from_lengths("long", [(1500, 300, 421), (700, 90, 33)], 4, 2, 128)
+    eo, el = _run_fwd(pack, 9)
+    assert eo <= TOL_O and el <= TOL_LSE, (eo, el)
+
+
+def test_empty_plan_is_a_noop():
+    plan = B.psa_plan([0], [], [], [], 4, 2, 64)
+    e = torch.empty((0, 4, 64), dtype=torch.bfloat16, device="cuda")
+    kv = torch.empty((0, 2, 64), dtype=torch.bfloat16, device="cuda")
+    o, lse = B.psa_fwd(plan, e, kv, kv)
+    assert o.numel() == 0 and lse.numel() == 0
+
+
+def test_misaligned_pointer_is_rejected():
+    pack = wl.config_pack(0)
+    plan = device_plan(pack)
+    q, k, v, _ = (t.cuda() for t in wl.attention_inputs(pack, 0))
+    buf = torch.empty(q.numel() + 8, dtype=torch.bfloat16, device="cuda")
+    q_bad = buf[1:1 + q.numel()].view_as(q)
+    with pytest.raises(B.PsaError) as e:
+        B.load_library()
+        B._check("psa_fwd", B.load_library().psa_fwd(plan._h, q_bad.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                                     q.data_ptr(), torch.empty(4, device="cuda").data_ptr(), None, None))
+    assert e.value.code == 4
