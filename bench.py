@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the prefix-shared DPO hot path on B200.
+
+One "step" is one pass of the whole path over one synthetic pack: psa_plan on the
+host, psa_fwd, psa_bwd, and dpo_logp over the pack's logits.  The headline metric
+is the useful TFLOP/s of attention forward + backward (14*d*Hq*U flops, U = the
+unmasked (q, kv) pairs per head) over the time of those two calls, measured with
+CUDA events inside the timed steps; packed tokens/s over the whole step and the
+gather's GB/s are reported beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..4] [--impl reference]
+
+N > 1 (launched through torch.distributed.run) runs N independent replicas: the
+path has no exchange step, so there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "psa_attention_fwd_bwd_useful_tflops"
+UNIT = "TFLOP/s"
+VOCAB = 128256            # logits width of the gather leg (bf16)
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    """Roofline denominators: the measured copy bandwidth and cuBLAS bf16 rate of
+    this machine's B200s if the driver left them, else an earlier measurement."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            self.proc.wait()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) >= 6 and r[2 + i] == "Active" for r in self.rows)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def oracle_sample(pack, steps, warmup, target="bench"):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload:
+    whole samples of the pack (attention is independent per sample) and one kv
+    group of 4 query heads.  Returns (useful TFLOP/s, description, cores, seconds per step)."""
+    import torch
+    from oracle import psa_oracle as orc
+    from paper_2410_20305_b200 import workloads as wl
+    order = np.argsort(pack.cu_seqlens[1:] - pack.cu_seqlens[:-1])
+    # the baseline leg takes the longest sample, the reference arm the shortest (it runs many steps)
+    s = int(order[-1] if target == "bench" else order[0])
+    P, C, R = int(pack.prefix_len[s]), int(pack.chosen_len[s]), int(pack.rejected_len[s])
+    sub = wl.pack_from_lengths("sample", [(P, C, R)], 4, 1, pack.head_dim)
+    q, k, v, d_o = (wl.to_f64(t) for t in wl.attention_inputs(sub, 2000, std=1.0))
+    mask = orc.packed_mask(sub.cu_seqlens, sub.prefix_len, sub.chosen_len, sub.rejected_len)
+    flops = 14.0 * pack.head_dim * 4 * orc.useful_pairs([P], [C], [R])
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        orc.attention_fwd(q, k, v, mask)
+        orc.attention_bwd(q, k, v, d_o, mask)
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+    sec = float(np.mean(times))
+    desc = "one sample of the pack (P=%d C=%d R=%d), 4 query heads / 1 kv head, fwd+bwd, dense fp64" % (P, C, R)
+    return flops / sec / 1e12, desc, torch.get_num_threads(), sec
+
+
+def run_reference(args, pack, rank):
+    """The reference arm: the CPU oracle on the machine's host cores, rank 0 only."""
+    if rank != 0:
+        return
+    val, desc, cores, sec = oracle_sample(pack, args.steps, args.warmup, target="reference")
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": pack.name, "sample": desc},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="psa", choices=["psa", "reference"])
+    ap.add_argument("--workload", type=int, default=1, help="1 llama3-8b, 2 long-prompt, 3 multi-turn, 4 short-many")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-paired", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    from paper_2410_20305_b200 import workloads as wl
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    pack = wl.config_pack(args.workload)
+    if args.impl == "reference":
+        return run_reference(args, pack, rank)
+
+    import torch
+    import torch.distributed as dist
+    import paper_2410_20305_b200 as psa
+    from paper_2410_20305_b200 import binding as B
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    T, Hq, Hkv, d = pack.total_tokens, pack.n_q_heads, pack.n_kv_heads, pack.head_dim
+    q, k, v, d_o = (t.to(dev) for t in wl.attention_inputs(pack, 2000 + args.workload, std=1.0))
+    gen = torch.Generator(device=dev).manual_seed(3000 + args.workload + rank)
+    logits = torch.empty((T, VOCAB), dtype=torch.bfloat16, device=dev)
+    for lo in range(0, T, 2048):   # N(0, variance 3), generated in slabs to bound the fp32 temporary
+        hi = min(T, lo + 2048)
+        logits[lo:hi] = (torch.randn((hi - lo, VOCAB), generator=gen, device=dev) * 3.0 ** 0.5).to(torch.bfloat16)
+    tok = torch.randint(0, VOCAB, (T,), generator=gen, device=dev, dtype=torch.int32).cpu().numpy()
+    targets, seg, fr, ft, fs = psa.logp_labels(tok, pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len)
+    i32 = lambda a: torch.as_tensor(np.asarray(a, dtype=np.int32)).to(dev)
+    targets, seg_d, fr, ft, fs = i32(targets), i32(seg), i32(fr), i32(ft), i32(fs)
+    n_seg = 2 * pack.n_samples
+    live_rows = int((seg >= 0).sum()) + int(((seg < 0)[fr.cpu().numpy()]).sum() if len(fr) else 0)
+
+    plan0 = B.psa_plan(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len, Hq, Hkv, d)
+    o = torch.empty_like(q); lse = torch.empty((Hq, T), dtype=torch.float32, device=dev)
+    dq = torch.empty_like(q); dk = torch.empty_like(k); dv = torch.empty_like(v)
+    ws = torch.empty(plan0.bwd_workspace_bytes, dtype=torch.uint8, device=dev)
+    logp = torch.empty(n_seg, dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    U = plan0.useful_pairs
+    flops_fwd, flops_bwd = 4.0 * d * Hq * U, 10.0 * d * Hq * U
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    n_total = args.warmup + args.steps
+    e_att0, e_att1, e_lp1 = [ev() for _ in range(n_total)], [ev() for _ in range(n_total)], [ev() for _ in range(n_total)]
+    k_fwd, k_bwd, k_lp = (ev(), ev()), (ev(), ev()), (ev(), ev())
+    kernel_ms = {"fwd": [], "bwd": [], "logp": []}
+
+    def step(i, timed):
+        plan = B.psa_plan(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len, Hq, Hkv, d)
+        e_att0[i].record()
+        B.psa_fwd(plan, q, k, v, o=o, lse=lse, status=status)
+        B.psa_bwd(plan, d_o, q, k, v, o, lse, dq=dq, dk=dk, dv=dv, workspace=ws, status=status)
+        e_att1[i].record()
+        B.dpo_logp(logits, targets, seg_d, n_seg, fr, ft, fs, out=logp, status=status)
+        e_lp1[i].record()
+        return plan
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # Per-kernel events (the library records them right around each main kernel) are read one
+    # step at a time in a separate short pass so that the timed region below stays free of syncs.
+    for i in range(args.warmup):
+        step(i, False)
+    sync_all()
+    for name, which, pair in (("fwd", 0, k_fwd), ("bwd", 1, k_bwd), ("logp", 2, k_lp)):
+        B.psa_profile_events(which, *pair)
+    for i in range(min(args.steps, 10)):
+        step(0, False)
+        torch.cuda.synchronize()
+        for name, pair in (("fwd", k_fwd), ("bwd", k_bwd), ("logp", k_lp)):
+            kernel_ms[name].append(pair[0].elapsed_time(pair[1]))
+    for which in range(3):
+        B.psa_profile_events(which)
+
+    sync_all()
+    t_start, t_stop = ev(), ev()
+    with ClockSampler(local_rank) as clocks:
+        t_start.record()
+        for i in range(args.warmup, n_total):
+            step(i, True)
+        t_stop.record()
+        sync_all()
+    step_ms = t_start.elapsed_time(t_stop) / args.steps
+    att_ms = float(np.mean([e_att0[i].elapsed_time(e_att1[i]) for i in range(args.warmup, n_total)]))
+    lp_ms = float(np.mean([e_att1[i].elapsed_time(e_lp1[i]) for i in range(args.warmup, n_total)]))
+    if int(status.item()) != 0:
+        raise SystemExit("device status word is %d: results invalid" % int(status.item()))
+
+    # ---- the same kernels on the unshared paired layout (2n causal sequences)
+    paired = None
+    if not args.no_paired and rank == 0:
+        pp = pack.paired()
+        pq, pk, pv, pdo = (t.to(dev) for t in wl.attention_inputs(pp, 2100 + args.workload))
+        pplan = B.psa_plan(pp.cu_seqlens, pp.prefix_len, pp.chosen_len, pp.rejected_len, Hq, Hkv, d)
+        po, plse = B.psa_fwd(pplan, pq, pk, pv)
+        pws = torch.empty(pplan.bwd_workspace_bytes, dtype=torch.uint8, device=dev)
+        pdq, pdk, pdv = B.psa_bwd(pplan, pdo, pq, pk, pv, po, plse, workspace=pws)
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(args.steps):
+            B.psa_fwd(pplan, pq, pk, pv, o=po, lse=plse)
+            B.psa_bwd(pplan, pdo, pq, pk, pv, po, plse, dq=pdq, dk=pdk, dv=pdv, workspace=pws)
+        b.record()
+        torch.cuda.synchronize()
+        p_ms = a.elapsed_time(b) / args.steps
+        paired = {"tokens": pp.total_tokens, "fwd_bwd_ms": p_ms, "speedup_shared_over_paired": p_ms / att_ms,
+                  "ideal_pair_ratio": pplan.useful_pairs / U, "token_ratio": pp.total_tokens / T}
+        del pq, pk, pv, pdo, po, plse, pws, pdq, pdk, pdv
+
+    # ---- end to end: pinned host inputs -> device -> fwd + bwd -> gradients and lse back on the host
+    e2e = None
+    if not args.no_e2e:
+        hq, hk, hv, hdo = (t.cpu().pin_memory() for t in (q, k, v, d_o))
+        h_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in (o, lse, dq, dk, dv)]
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hdo))
+        d2h = sum(t.numel() * t.element_size() for t in h_out)
+
+        def e2e_step():
+            q.copy_(hq, non_blocking=True); k.copy_(hk, non_blocking=True)
+            v.copy_(hv, non_blocking=True); d_o.copy_(hdo, non_blocking=True)
+            plan = B.psa_plan(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len, Hq, Hkv, d)
+            B.psa_fwd(plan, q, k, v, o=o, lse=lse)
+            B.psa_bwd(plan, d_o, q, k, v, o, lse, dq=dq, dk=dk, dv=dv, workspace=ws)
+            for h, t in zip(h_out, (o, lse, dq, dk, dv)):
+                h.copy_(t, non_blocking=True)
+            torch.cuda.synchronize()
+            return plan
+        for _ in range(3):
+            e2e_step()
+        sync_all()
+        t0 = time.perf_counter()
+        n_e2e = max(3, min(args.steps, 10))
+        for _ in range(n_e2e):
+            e2e_step()
+        sync_all()
+        e2e_ms = (time.perf_counter() - t0) * 1e3 / n_e2e
+        e2e = {"value": (flops_fwd + flops_bwd) / e2e_ms / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    # ---- max over ranks (replicas): whole-job value = sum of the replicas' useful flops / slowest time
+    times = torch.tensor([step_ms, att_ms, lp_ms, e2e["ms_per_step"] if e2e else 0.0], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    step_ms, att_ms, lp_ms, e2e_ms_max = (float(x) for x in times.cpu())
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    value = world * (flops_fwd + flops_bwd) / att_ms / 1e9
+    bwd_ms, fwd_ms, klp_ms = (float(np.mean(kernel_ms[n])) for n in ("bwd", "fwd", "logp"))
+    bwd_tflops = flops_bwd / bwd_ms / 1e9
+    logp_bytes = live_rows * VOCAB * 2 + 8 * live_rows + 4 * n_seg
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": pack.name, "pack_len": pack.pack_len, "total_tokens": T, "n_samples": pack.n_samples,
+                   "n_q_heads": Hq, "n_kv_heads": Hkv, "head_dim": d, "useful_pairs_per_head": U,
+                   "live_tiles": plan0.live_tiles, "partial_tiles": plan0.partial_tiles, "logits": [T, VOCAB],
+                   "l2": "inputs larger than L2 (q, o, dO, dq are 133 MB each; logits %.1f GB)" % (T * VOCAB * 2 / 1e9),
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "attention_fwd_bwd_ms": att_ms,
+        "pct_of_bf16_peak": {"measured": value / world / peaks["bf16_tflops"], "nominal": value / world / NOMINAL_BF16_TFLOPS,
+                             "peak_source": peaks["source"]},
+        "tokens_per_s": world * T / (step_ms * 1e-3),
+        "attention_tokens_per_s": world * T / (att_ms * 1e-3),
+        "kernels": {"psa_fwd_ms": fwd_ms, "psa_fwd_tflops": flops_fwd / fwd_ms / 1e9,
+                    "psa_bwd_main_ms": bwd_ms, "psa_bwd_main_tflops": bwd_tflops,
+                    "dpo_logp_ms": klp_ms, "dpo_logp_gbs": logp_bytes / klp_ms / 1e6,
+                    "dpo_logp_frac_of_hbm": {"measured": logp_bytes / klp_ms / 1e6 / peaks["hbm_gbs"],
+                                             "nominal": logp_bytes / klp_ms / 1e6 / NOMINAL_HBM_GBS},
+                    "dpo_logp_live_rows": live_rows, "dpo_logp_step_ms": lp_ms},
+        "roofline": {"kernel": "psa_bwd_kernel<128>", "bound": "tensor", "achieved": bwd_tflops,
+                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": bwd_tflops / peaks["bf16_tflops"],
+                     "peak_kind": "burst bf16 cuBLAS, of " + peaks["source"], "traffic": None},
+        "clocks": clocks.summary(),
+        "gpu_launches": args.steps * 5,
+        "paired_layout": paired,
+        "paper_context": "paper reports 1.1-1.5x (1.3-1.6x with packing) end-to-end training speedups on 8xH100; context, not the target",
+    }
+    if e2e:
+        e2e["value"] = world * (flops_fwd + flops_bwd) / e2e_ms_max / 1e9
+        e2e["ms_per_step"] = e2e_ms_max
+        line["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        val, desc, cores, sec = oracle_sample(pack, 1, 0)
+        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                                "seconds": sec}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -185,6 +185,19 @@ psa_status_t dpo_logp(const void* logits, int32_t logits_dtype, int64_t n_rows, 
                       const int32_t* fork_segments, int32_t n_forks, int32_t n_segments,
                       float* out, int32_t* device_status, void* stream);
 
+/*
+ * psa_profile_events -- measurement aid, no counterpart in the paper.  Registers a
+ * pair of cudaEvent_t (passed as void*) that the next calls record on their stream
+ * immediately before and after one chosen kernel, so that a benchmark can time that
+ * kernel alone while it runs inside a whole step.
+ *   which   0 = the psa_fwd kernel, 1 = the main psa_bwd kernel (without the
+ *           delta / clear / convert helpers), 2 = the dpo_logp kernel
+ *   start, stop   events created with timing enabled; pass NULL, NULL to unregister.
+ * Process-global and not thread-safe; the events must outlive the calls they time.
+ * Errors: INVALID_ARG (bad `which`, or only one of the two events given).
+ */
+psa_status_t psa_profile_events(int32_t which, void* start, void* stop);
+
 #ifdef __cplusplus
 }
 #endif

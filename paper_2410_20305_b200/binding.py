@@ -22,7 +22,7 @@ PSA_DEVSTAT_WAIT_EXPIRED, PSA_DEVSTAT_BAD_TARGET, PSA_DEVSTAT_BAD_SEGMENT = 1, 2
 
 EXPORTED_SYMBOLS = (
     "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
-    "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp",
+    "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp", "psa_profile_events",
 )
 
 
@@ -59,6 +59,7 @@ def load_library():
     lib.psa_plan_export.argtypes = [vp, i32, vp, vp]
     lib.psa_fwd.argtypes = [vp] * 8
     lib.psa_bwd.argtypes = [vp] * 13
+    lib.psa_profile_events.argtypes = [i32, vp, vp]
     lib.dpo_logp.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     for name in EXPORTED_SYMBOLS:
         if name != "psa_status_string":
@@ -202,3 +203,15 @@ def dpo_logp(logits, targets, segment_ids, n_segments, fork_rows=None, fork_targ
                                                _ptr(fork_segments), n_forks, n_segments, _ptr(out), _ptr(status),
                                                _stream(stream)))
     return out
+
+
+def psa_profile_events(which, start=None, stop=None):
+    """Registers (or, with None, removes) a pair of torch.cuda.Event recorded right
+    before and after one kernel: 0 = psa_fwd, 1 = main psa_bwd kernel, 2 = dpo_logp."""
+    if start is not None:
+        # torch creates the underlying cudaEvent lazily, on the first record
+        start.record()
+        stop.record()
+    a = C.c_void_p(0) if start is None else C.c_void_p(start.cuda_event)
+    b = C.c_void_p(0) if stop is None else C.c_void_p(stop.cuda_event)
+    _check("psa_profile_events", load_library().psa_profile_events(which, a, b))

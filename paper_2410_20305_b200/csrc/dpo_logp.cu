@@ -11,6 +11,7 @@
 #include <cmath>
 
 #include "psa.h"
+#include "psa_internal.h"
 
 namespace psa {
 namespace {
@@ -179,6 +180,7 @@ extern "C" psa_status_t dpo_logp(const void* logits, int32_t logits_dtype, int64
     return PSA_ERR_CUDA;
   if (n_rows == 0) return PSA_OK;
   const unsigned grid = unsigned(n_rows);
+  psa::ProfileScope prof(2, stream);
   if (logits_dtype == PSA_DTYPE_F32)
     psa::dpo_logp_kernel<float, 4><<<grid, psa::kLogpThreads, 0, st>>>(
         static_cast<const float*>(logits), vocab, row_stride, targets, segment_ids, fork_rows, fork_targets,

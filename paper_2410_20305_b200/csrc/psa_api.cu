@@ -31,3 +31,19 @@ extern "C" psa_status_t psa_bwd(const psa_plan_t* plan, const void* d_o, const v
     return PSA_ERR_ALIGNMENT;
   return psa::launch_bwd(plan, d_o, q, k, v, o, lse, dq, dk, dv, workspace, device_status, stream);
 }
+
+namespace psa {
+ProfileEvents g_profile[3] = {{nullptr, nullptr}, {nullptr, nullptr}, {nullptr, nullptr}};
+ProfileScope::ProfileScope(int which, void* s) : ev(g_profile[which]), stream(s) {
+  if (ev.start) cudaEventRecord(cudaEvent_t(ev.start), cudaStream_t(stream));
+}
+ProfileScope::~ProfileScope() {
+  if (ev.stop) cudaEventRecord(cudaEvent_t(ev.stop), cudaStream_t(stream));
+}
+}  // namespace psa
+
+extern "C" psa_status_t psa_profile_events(int32_t which, void* start, void* stop) {
+  if (which < 0 || which > 2 || ((start == nullptr) != (stop == nullptr))) return PSA_ERR_INVALID_ARG;
+  psa::g_profile[which] = psa::ProfileEvents{start, stop};
+  return PSA_OK;
+}

@@ -6,6 +6,7 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -174,18 +175,29 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t
   d |= uint64_t(2) << 61;  // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, dense.
-__host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, bool a_mn_major, bool b_mn_major) {
+// Instruction descriptor of a dense 16-bit x 16-bit -> fp32 UMMA.  A and B carry separate
+// format fields (kF16 or kBF16) but they must be equal: an fp16 A with a bf16 B is rejected
+// by the hardware as an illegal instruction.
+constexpr uint32_t kF16 = 0, kBF16 = 1;
+__host__ __device__ constexpr uint32_t umma_idesc(int M, int N, uint32_t a_fmt, uint32_t b_fmt, bool a_mn_major,
+                                                  bool b_mn_major) {
   return (1u << 4)                       // D is fp32
-         | (1u << 7) | (1u << 10)        // A, B are bf16
+         | (a_fmt << 7) | (b_fmt << 10)
          | (uint32_t(a_mn_major) << 15) | (uint32_t(b_mn_major) << 16)
          | (uint32_t(N >> 3) << 17) | (uint32_t(M >> 4) << 24);
+}
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, bool a_mn_major, bool b_mn_major) {
+  return umma_idesc(M, N, kBF16, kBF16, a_mn_major, b_mn_major);
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);

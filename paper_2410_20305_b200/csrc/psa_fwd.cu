@@ -125,8 +125,8 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_wait(bar(BAR_Q_FULL), 0, wctx);
       for (int it = 0; it < n_it; ++it) {
         mbar_wait(bar(BAR_K_FULL), it & 1, wctx);
-        // The S columns are also where P_{it-1} lives: wait until the previous P V has read it.
-        if (it > 0) mbar_wait(bar(BAR_O_FULL), (it - 1) & 1, wctx);
+        // The S columns are also where P_{it-1} lives.  UMMAs issued by one thread execute in
+        // issue order, so this S = Q K^T cannot overwrite P before the previous P V has read it.
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
@@ -280,12 +280,8 @@ psa_status_t launch_fwd_t(const psa_plan_t* plan, const void* q, const void* k, 
   if (!make_tile_map_bf16(&tm_q, q, plan->T, plan->Hq, D) || !make_tile_map_bf16(&tm_k, k, plan->T, plan->Hkv, D) ||
       !make_tile_map_bf16(&tm_v, v, plan->T, plan->Hkv, D))
     return PSA_ERR_CUDA;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(psa_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kRequest) != cudaSuccess)
-      return PSA_ERR_CUDA;
-    attr_done = true;
-  }
+  if (cudaFuncSetAttribute(psa_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kRequest) != cudaSuccess)
+    return PSA_ERR_CUDA;
   FwdParams prm;
   prm.tiles = plan->d_q_tiles;
   prm.entries = plan->d_fwd_entries;
@@ -297,7 +293,10 @@ psa_status_t launch_fwd_t(const psa_plan_t* plan, const void* q, const void* k, 
   prm.Hkv = plan->Hkv;
   prm.scale_log2 = plan->scale * 1.4426950408889634f;
   const unsigned grid = unsigned(plan->q_tiles.size()) * unsigned(plan->Hq);
-  psa_fwd_kernel<D><<<grid, kFwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, prm);
+  {
+    ProfileScope prof(0, stream);
+    psa_fwd_kernel<D><<<grid, kFwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, prm);
+  }
   return cudaGetLastError() == cudaSuccess ? PSA_OK : PSA_ERR_CUDA;
 }
 

@@ -42,6 +42,15 @@ struct psa_plan {
 };
 
 namespace psa {
+// Optional event pairs recorded around one kernel (see psa_profile_events).
+struct ProfileEvents { void* start; void* stop; };
+extern ProfileEvents g_profile[3];
+struct ProfileScope {  // records start now and stop at scope exit, if registered
+  ProfileEvents ev; void* stream;
+  ProfileScope(int which, void* s);
+  ~ProfileScope();
+};
+
 // Workspace layout of psa_bwd (byte offsets, each 256-aligned).
 struct BwdWorkspace {
   size_t dq_accum_off, dq_accum_bytes;  // fp32 [T, Hq, d]

@@ -36,6 +36,30 @@ def max_abs(a, b):
     return float(d.max())
 
 
+def half_ulp_bf16(ref):
+    """Half a bf16 unit in the last place at each reference value (bf16 keeps 8
+    significant bits): the error a correctly rounded bf16 output may carry."""
+    a = np.abs(np.asarray(ref, dtype=np.float64))
+    e = np.floor(np.log2(np.maximum(a, 2.0 ** -126)))
+    return 2.0 ** (e - 8)
+
+
+def grad_errors(a, ref):
+    """For a bf16 gradient tensor returns (raw max abs error, max abs error on the
+    elements with |ref| < 2, max of error minus the bf16 half-ulp at the reference).
+    The gate of 1e-2 is applied to the last two: where |ref| >= 2 the rounding of
+    the exact value to bf16 alone can exceed 1e-2 (half an ulp is 0.0156 in [4, 8)),
+    so there the gate bounds the error in excess of that rounding."""
+    a = a.detach().to("cpu").to(torch.float64).numpy()
+    assert np.isfinite(a).all(), "non-finite values in the GPU result"
+    if a.size == 0:
+        return 0.0, 0.0, 0.0
+    err = np.abs(a - ref)
+    small = np.abs(ref) < 2.0
+    return (float(err.max()), float(err[small].max(initial=0.0)),
+            float((err - half_ulp_bf16(ref)).max()))
+
+
 def read_status(status):
     torch.cuda.synchronize()
     return int(status.item())
