@@ -116,7 +116,9 @@ psa_status_t psa_plan_stats(const psa_plan_t* plan, int64_t* total_tokens,
  * rejected_start, entry_offset, entry_count }, where row0 is the packed-row
  * index of the tile's first row, local0 = row0 - sample_start, and
  * chosen_start / rejected_start are relative to sample_start.  An entry is
- * (tile_index_within_sample << 1) | needs_mask.
+ * (tile_index_within_sample << 2) | (precise << 1) | needs_mask, where `precise`
+ * marks query tiles holding a row with fewer than 128 visible keys: for those the
+ * kernels keep the probabilities (and dS) as a sum of two bf16 terms.
  * `tiles` is host int32 [n_tiles*8], `entries` host int32 [n_entries].
  */
 psa_status_t psa_plan_counts(const psa_plan_t* plan, int32_t direction,

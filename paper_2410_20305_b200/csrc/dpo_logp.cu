@@ -189,5 +189,5 @@ extern "C" psa_status_t dpo_logp(const void* logits, int32_t logits_dtype, int64
     psa::dpo_logp_kernel<__nv_bfloat16, 4><<<grid, psa::kLogpThreads, 0, st>>>(
         static_cast<const __nv_bfloat16*>(logits), vocab, row_stride, targets, segment_ids, fork_rows, fork_targets,
         fork_segments, n_forks, n_segments, out, device_status);
-  return cudaGetLastError() == cudaSuccess ? PSA_OK : PSA_ERR_CUDA;
+  return psa::check_last_cuda_error("dpo_logp launch");
 }

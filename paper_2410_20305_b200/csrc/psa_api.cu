@@ -1,6 +1,9 @@
 // extern "C" entry points psa_fwd / psa_bwd: argument validation, then the launchers.
 #include <cuda_runtime.h>
 
+#include <cstdio>
+#include <cstdlib>
+
 #include "psa_internal.h"
 
 namespace {
@@ -33,6 +36,13 @@ extern "C" psa_status_t psa_bwd(const psa_plan_t* plan, const void* d_o, const v
 }
 
 namespace psa {
+psa_status_t check_last_cuda_error(const char* where) {
+  const cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) return PSA_OK;
+  if (std::getenv("PSA_DEBUG")) std::fprintf(stderr, "libpsa: %s: %s\n", where, cudaGetErrorString(e));
+  return PSA_ERR_CUDA;
+}
+
 ProfileEvents g_profile[3] = {{nullptr, nullptr}, {nullptr, nullptr}, {nullptr, nullptr}};
 ProfileScope::ProfileScope(int which, void* s) : ev(g_profile[which]), stream(s) {
   if (ev.start) cudaEventRecord(cudaEvent_t(ev.start), cudaStream_t(stream));

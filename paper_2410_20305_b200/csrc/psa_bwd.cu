@@ -23,6 +23,7 @@
 #include <cuda_runtime.h>
 
 #include <cmath>
+#include <type_traits>
 
 #include "psa_device.cuh"
 #include "psa_internal.h"
@@ -40,7 +41,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 
 struct BwdParams {
   const TileRec* tiles;     // key tiles
-  const int32_t* entries;   // (query tile << 1) | needs_mask
+  const int32_t* entries;   // (query tile << 2) | (precise << 1) | needs_mask
   const float* lse;         // [Hq, T]
   const float* delta;       // [Hq, T]
   float* dq_accum;          // [T, Hq, D] fp32
@@ -71,7 +72,7 @@ struct BwdSmem {
 
 enum {
   B_KV_FULL = 0, B_Q_FULL0, B_Q_FULL1, B_DO_FULL0, B_DO_FULL1, B_QDO_EMPTY0, B_QDO_EMPTY1,
-  B_S_FULL, B_DP_FULL, B_P_FULL, B_DS_FULL, B_DQ_FULL, B_DQ_EMPTY, B_COUNT
+  B_S_FULL, B_DP_FULL, B_P_FULL, B_DS_FULL, B_DS_EMPTY, B_DQ_FULL, B_DQ_EMPTY, B_COUNT
 };
 
 __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
@@ -147,7 +148,7 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       for (int it = 0; it < n_it; ++it) {
         const int st = it & 1;
         const int h = head_of(it);
-        const int qrow = rec.ds + (entry_of(it) >> 1) * kTile;
+        const int qrow = rec.ds + (entry_of(it) >> 2) * kTile;
         if (it >= 2) mbar_wait(bar(B_QDO_EMPTY0 + st), ((it >> 1) - 1) & 1, wctx);
         mbar_expect_tx(bar(B_Q_FULL0 + st), L::kTileBytes);
         for (int s = 0; s < L::kSub; ++s) tma_load_3d(sQ(st) + s * L::kSubBytes, &tm_q, s * 64, h, qrow, bar(B_Q_FULL0 + st));
@@ -164,8 +165,11 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       constexpr uint32_t idesc_dk = umma_idesc_bf16(kTile, D, false, true);       // dS^T (K-major) x Q (MN-major)
       constexpr uint32_t idesc_dq = umma_idesc_bf16(kTile, D, true, true);        // dS (MN-major) x K (MN-major)
       mbar_wait(bar(B_KV_FULL), 0, wctx);
+      uint32_t ds_ph = 0;  // running parity of B_DS_FULL (it completes twice in a PRECISE iteration)
       for (int it = 0; it < n_it; ++it) {
         const int st = it & 1, ph = (it >> 1) & 1;
+        // PRECISE tiles carry P^T and dS^T as two bf16 terms each.
+        const int n_terms = (entry_of(it) & 2) ? 2 : 1;
         // S^T = K Q^T.  (Its columns held P^T of the previous iteration; the dV product that
         // read it was issued earlier by this thread and UMMAs execute in issue order.)
         mbar_wait(bar(B_Q_FULL0 + st), ph, wctx);
@@ -191,21 +195,30 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // dV += P^T dO   (reduction over the 128 query rows, 16 per instruction)
         mbar_wait(bar(B_P_FULL), it & 1, wctx);
         tc_fence_after();
+        for (int term = 0; term < n_terms; ++term) {   // second term: columns [64,128) of the S region
 #pragma unroll
-        for (int kk = 0; kk < kTile / 16; ++kk)
-          umma_ts(tmem + kColDV, tmem + kColS + kk * 8, smem_desc_sw128(sDO(st) + kk * 2048, L::kSubBytes, 1024),
-                  idesc_dv, (it > 0) || (kk > 0));
-        // dK += dS^T Q ; dQ = dS K
-        mbar_wait(bar(B_DS_FULL), it & 1, wctx);
-        tc_fence_after();
+          for (int kk = 0; kk < kTile / 16; ++kk)
+            umma_ts(tmem + kColDV, tmem + kColS + term * 64 + kk * 8,
+                    smem_desc_sw128(sDO(st) + kk * 2048, L::kSubBytes, 1024), idesc_dv,
+                    (it > 0) || (kk > 0) || (term > 0));
+        }
+        // dK += dS^T Q ; dQ = dS K.  The two terms of a PRECISE tile pass through the one
+        // shared-memory buffer one after the other.
+        for (int term = 0; term < n_terms; ++term) {
+          mbar_wait(bar(B_DS_FULL), ds_ph, wctx);
+          ds_ph ^= 1;
+          tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < kTile / 16; ++kk)
-          umma_ss(tmem + kColDK, smem_desc_sw128(sDS + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
-                  smem_desc_sw128(sQ(st) + kk * 2048, L::kSubBytes, 1024), idesc_dk, (it > 0) || (kk > 0));
+          for (int kk = 0; kk < kTile / 16; ++kk)
+            umma_ss(tmem + kColDK, smem_desc_sw128(sDS + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
+                    smem_desc_sw128(sQ(st) + kk * 2048, L::kSubBytes, 1024), idesc_dk,
+                    (it > 0) || (kk > 0) || (term > 0));
 #pragma unroll
-        for (int kk = 0; kk < kTile / 16; ++kk)
-          umma_ss(tmem + kColDP, smem_desc_sw128(sDS + kk * 2048, 16384, 1024),
-                  smem_desc_sw128(sK + kk * 2048, L::kSubBytes, 1024), idesc_dq, kk > 0);
+          for (int kk = 0; kk < kTile / 16; ++kk)
+            umma_ss(tmem + kColDP, smem_desc_sw128(sDS + kk * 2048, 16384, 1024),
+                    smem_desc_sw128(sK + kk * 2048, L::kSubBytes, 1024), idesc_dq, (kk > 0) || (term > 0));
+          if (term + 1 < n_terms) umma_commit(bar(B_DS_EMPTY));
+        }
         umma_commit(bar(B_DQ_FULL));
         umma_commit(bar(B_QDO_EMPTY0 + st));
       }
@@ -224,7 +237,7 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const float cl = prm.scale_log2;
 
     auto load_stats = [&](int it, float& l2, float& dl) {
-      const int64_t qrow = int64_t(rec.ds) + (entry_of(it) >> 1) * kTile + ct;
+      const int64_t qrow = int64_t(rec.ds) + (entry_of(it) >> 2) * kTile + ct;
       l2 = 0.f;
       dl = 0.f;
       if (qrow < prm.T) {
@@ -241,10 +254,16 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
     named_bar_sync(1, 128);
 
-    for (int it = 0; it < n_it; ++it) {
+    uint32_t dse_ph = 0;  // running parity of B_DS_EMPTY
+
+    // One iteration = one (query head, query tile).  Two instantiations: PRECISE tiles carry
+    // P^T and dS^T as two bf16 terms (and recompute delta exactly for a sample's first query
+    // tile); keeping that out of the common instantiation keeps its register use down.
+    auto iteration = [&](int it, auto precise_tag) {
+      constexpr bool kPrecise = decltype(precise_tag)::value;
       const int st = it & 1;
       const int e = entry_of(it);
-      const int q0 = (e >> 1) * kTile;
+      const int q0 = (e >> 2) * kTile;
       float nl2 = 0.f, ndl = 0.f;
       if (it + 1 < n_it) load_stats(it + 1, nl2, ndl);
 
@@ -283,6 +302,11 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = pack_bf16x2(p[ch * 64 + 2 * i], p[ch * 64 + 2 * i + 1]);
         tmem_st32(tmem + lane_base + kColS + ch * 32, v);
+        if constexpr (kPrecise) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) v[i] = pack_bf16x2_residual(p[ch * 64 + 2 * i], p[ch * 64 + 2 * i + 1], v[i]);
+          tmem_st32(tmem + lane_base + kColS + 64 + ch * 32, v);
+        }
       }
       tc_wait_st();
       tc_fence_before();
@@ -292,7 +316,42 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       // iteration completed after the previous iteration's dK / dQ products.
       mbar_wait(bar(B_DP_FULL), it & 1, wctx);
       tc_fence_after();
+      if constexpr (kPrecise) {
+        if ((e >> 2) == 0) {
+          // Rows of a sample's first query tile see only this key tile, and they are the rows
+          // with few keys, where delta = dO . O computed from the bf16-rounded O is the largest
+          // error left.  Recompute it exactly here:  delta_i = sum_j P_ij dP_ij  (fp32).
+          // Column sums over the 128 key rows: transpose-reduce inside each warp, then add the
+          // four warps through the (still unused) dS buffer.
+          float* scratch = reinterpret_cast<float*>(smem_raw + L::kDS);
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            uint32_t v[32];
+            tmem_ld32(tmem + lane_base + kColDP + ch * 32, v);
+            tc_wait_ld();
+            float t[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) t[i] = p[ch * 32 + i] * __uint_as_float(v[i]);
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) {
+              const bool up = (lane & off) != 0;
+#pragma unroll
+              for (int kq = 0; kq < off; ++kq) {
+                const float send = up ? t[kq] : t[kq + off];
+                const float keep = up ? t[kq + off] : t[kq];
+                t[kq] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+              }
+            }
+            scratch[quarter * kTile + ch * 32 + lane] = t[0];   // lane l now holds column ch*32 + l
+          }
+          named_bar_sync(1, 128);
+          const float dsum = scratch[ct] + scratch[kTile + ct] + scratch[2 * kTile + ct] + scratch[3 * kTile + ct];
+          s_delta[st * kTile + ct] = dsum;
+          named_bar_sync(1, 128);
+        }
+      }
       const float4* d4 = reinterpret_cast<const float4*>(s_delta + st * kTile);
+      uint32_t ds_lo[kPrecise ? 64 : 1];  // second bf16 term of dS^T
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
         uint32_t v[32];
@@ -308,6 +367,10 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           const float a3 = p[ch * 32 + 4 * i + 3] * (__uint_as_float(v[4 * i + 3]) - dl.w);
           w[2 * i] = pack_bf16x2(a0, a1);
           w[2 * i + 1] = pack_bf16x2(a2, a3);
+          if constexpr (kPrecise) {
+            ds_lo[ch * 16 + 2 * i] = pack_bf16x2_residual(a0, a1, w[2 * i]);
+            ds_lo[ch * 16 + 2 * i + 1] = pack_bf16x2_residual(a2, a3, w[2 * i + 1]);
+          }
         }
         // Row r of the 128 x 128 bf16 tile: 64-column half (ch >> 1), 16-byte chunks
         // (ch & 1) * 4 .. + 3, each stored at chunk index XOR (r & 7)  (128-byte swizzle).
@@ -321,10 +384,31 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(bar(B_DS_FULL));
+      if constexpr (kPrecise) {
+        // second term: same buffer, once the products of the first term have read it
+        mbar_wait(bar(B_DS_EMPTY), dse_ph, wctx);
+        dse_ph ^= 1;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          const uint32_t row_addr = sDS + (ch >> 1) * 16384 + r * 128;
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) {
+            const uint32_t chunk = uint32_t((ch & 1) * 4 + c4) ^ uint32_t(r & 7);
+            st_shared_v4(row_addr + chunk * 16, ds_lo[ch * 16 + 4 * c4], ds_lo[ch * 16 + 4 * c4 + 1],
+                         ds_lo[ch * 16 + 4 * c4 + 2], ds_lo[ch * 16 + 4 * c4 + 3]);
+          }
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(bar(B_DS_FULL));
+      }
 
       s_lse[(st ^ 1) * kTile + ct] = nl2;
       s_delta[(st ^ 1) * kTile + ct] = ndl;
       named_bar_sync(1, 128);
+    };
+    for (int it = 0; it < n_it; ++it) {
+      if (entry_of(it) & 2) iteration(it, std::true_type{});
+      else iteration(it, std::false_type{});
     }
 
     // ---- epilogue: dV, dK (scaled) -> bf16
@@ -363,7 +447,7 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t lane_base = uint32_t(quarter * 32) << 16;
     const float sc = prm.scale;
     for (int it = 0; it < n_it; ++it) {
-      const int q0 = (entry_of(it) >> 1) * kTile;
+      const int q0 = (entry_of(it) >> 2) * kTile;
       const bool valid = q0 + r < rec.len;
       float* dst_row = prm.dq_accum + ((int64_t(rec.ds) + q0 + r) * prm.Hq + head_of(it)) * D;
       mbar_wait(bar(B_DQ_FULL), it & 1, wctx);
@@ -484,7 +568,7 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
     psa_bwd_convert_kernel<<<unsigned((n_vec4 + 255) / 256), 256, 0, stream>>>(
         reinterpret_cast<const float4*>(dq_accum), static_cast<uint2*>(dq), n_vec4);
   }
-  return cudaGetLastError() == cudaSuccess ? PSA_OK : PSA_ERR_CUDA;
+  return check_last_cuda_error("psa_bwd launch");
 }
 
 }  // namespace

@@ -199,6 +199,12 @@ __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
   __half2 v = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+// Residual pair of a packed bf16 pair: pack(lo - bf16(lo), hi - bf16(hi)), so that the two
+// packed words together carry about 16 significant bits of each value.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi);
+__device__ __forceinline__ uint32_t pack_bf16x2_residual(float lo, float hi, uint32_t packed) {
+  return pack_bf16x2(lo - __uint_as_float(packed << 16), hi - __uint_as_float(packed & 0xffff0000u));
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);

@@ -13,6 +13,7 @@
 #include <cuda_runtime.h>
 
 #include <cmath>
+#include <type_traits>
 
 #include "psa_device.cuh"
 #include "psa_internal.h"
@@ -107,7 +108,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_expect_tx(bar(BAR_Q_FULL), L::kTileBytes);
       for (int s = 0; s < L::kSub; ++s) tma_load_3d(sQ + s * L::kSubBytes, &tm_q, s * 64, h, rec.row0, bar(BAR_Q_FULL));
       for (int it = 0; it < n_it; ++it) {
-        const int krow = rec.ds + (ent[it] >> 1) * kTile;
+        const int krow = rec.ds + (ent[it] >> 2) * kTile;
         if (it > 0) mbar_wait(bar(BAR_K_EMPTY), (it - 1) & 1, wctx);
         mbar_expect_tx(bar(BAR_K_FULL), L::kTileBytes);
         for (int s = 0; s < L::kSub; ++s) tma_load_3d(sK + s * L::kSubBytes, &tm_k, s * 64, hk, krow, bar(BAR_K_FULL));
@@ -139,11 +140,15 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         mbar_wait(bar(BAR_V_FULL), it & 1, wctx);
         mbar_wait(bar(BAR_P_FULL), it & 1, wctx);
         tc_fence_after();
+        // PRECISE tiles carry P as two bf16 terms: columns [0,64) and [64,128) of the S region.
+        const int n_terms = (ent[it] & 2) ? 2 : 1;
+        for (int term = 0; term < n_terms; ++term) {
 #pragma unroll
-        for (int kk = 0; kk < kTile / 16; ++kk) {
-          // A: 16 keys of P = 8 TMEM columns (two bf16 per column).  B: 16 key rows of V.
-          umma_ts(tmem + kColO, tmem + kColS + kk * 8, smem_desc_sw128(sV + kk * 2048, L::kSubBytes, 1024), idesc_o,
-                  (it > 0) || (kk > 0));
+          for (int kk = 0; kk < kTile / 16; ++kk) {
+            // A: 16 keys of P = 8 TMEM columns (two bf16 per column).  B: 16 key rows of V.
+            umma_ts(tmem + kColO, tmem + kColS + term * 64 + kk * 8,
+                    smem_desc_sw128(sV + kk * 2048, L::kSubBytes, 1024), idesc_o, (it > 0) || (kk > 0) || (term > 0));
+          }
         }
         umma_commit(bar(BAR_V_EMPTY));
         umma_commit(bar(BAR_O_FULL));
@@ -162,7 +167,8 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
     for (int it = 0; it < n_it; ++it) {
       const int e = ent[it];
-      const int k0 = (e >> 1) * kTile;
+      const int k0 = (e >> 2) * kTile;
+      const bool precise = (e & 2) != 0;
       mbar_wait(bar(BAR_S_FULL), it & 1, wctx);
       tc_fence_after();
       float s[kTile];
@@ -214,18 +220,26 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       const float mc = (m_run == -INFINITY) ? 0.f : m_run * c;
       float sum = 0.f;
+      // P -> bf16 over the S columns ([0,64)); PRECISE tiles also store the rounding residual as a
+      // second bf16 term in columns [64,128).  Two instantiations keep the common path lean.
+      auto write_p = [&](auto precise_tag) {
+        constexpr bool kPrecise = decltype(precise_tag)::value;
 #pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t v[32];
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t v[32], vr[kPrecise ? 32 : 1];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float p0 = ex2_approx(fmaf(s[ch * 64 + 2 * i], c, -mc));
-          const float p1 = ex2_approx(fmaf(s[ch * 64 + 2 * i + 1], c, -mc));
-          sum += p0 + p1;
-          v[i] = pack_bf16x2(p0, p1);
+          for (int i = 0; i < 32; ++i) {
+            const float p0 = ex2_approx(fmaf(s[ch * 64 + 2 * i], c, -mc));
+            const float p1 = ex2_approx(fmaf(s[ch * 64 + 2 * i + 1], c, -mc));
+            sum += p0 + p1;
+            v[i] = pack_bf16x2(p0, p1);
+            if constexpr (kPrecise) vr[i] = pack_bf16x2_residual(p0, p1, v[i]);
+          }
+          tmem_st32(tmem + lane_base + kColS + ch * 32, v);
+          if constexpr (kPrecise) tmem_st32(tmem + lane_base + kColS + 64 + ch * 32, vr);
         }
-        tmem_st32(tmem + lane_base + kColS + ch * 32, v);
-      }
+      };
+      if (precise) write_p(std::true_type{}); else write_p(std::false_type{});
       l_run += sum;
       tc_wait_st();
       tc_fence_before();
@@ -297,7 +311,7 @@ psa_status_t launch_fwd_t(const psa_plan_t* plan, const void* q, const void* k, 
     ProfileScope prof(0, stream);
     psa_fwd_kernel<D><<<grid, kFwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, prm);
   }
-  return cudaGetLastError() == cudaSuccess ? PSA_OK : PSA_ERR_CUDA;
+  return check_last_cuda_error("psa_fwd launch");
 }
 
 }  // namespace

@@ -42,6 +42,10 @@ struct psa_plan {
 };
 
 namespace psa {
+// Returns PSA_OK if no CUDA error is pending, else PSA_ERR_CUDA; with PSA_DEBUG set in the
+// environment the CUDA error string is written to stderr.
+psa_status_t check_last_cuda_error(const char* where);
+
 // Optional event pairs recorded around one kernel (see psa_profile_events).
 struct ProfileEvents { void* start; void* stop; };
 extern ProfileEvents g_profile[3];

@@ -50,6 +50,16 @@ int classify(int i, int j, int len, int cs, int rs, bool bwd) {
   return partial ? 2 : 1;
 }
 
+// A query tile is PRECISE when one of its rows sees fewer than 128 keys.  Such rows
+// have large probabilities, whose bf16 rounding dominates the error of dK and dV;
+// the kernels carry P and dS of these tiles as a sum of two bf16 terms.
+bool precise_rows(int i, int len, int cs, int rs) {
+  if (i == 0) return true;                          // row 0 sees one key
+  const int q0 = i * kTile, q1 = std::min(q0 + kTile, len);
+  const int q = std::max(q0, rs);                   // first rejected row of the tile, if any
+  return q < q1 && cs + (q - rs + 1) < kTile;       // it sees the prompt and q - rs + 1 own keys
+}
+
 }  // namespace
 }  // namespace psa
 
@@ -111,7 +121,7 @@ extern "C" psa_status_t psa_plan(const int32_t* cu_seqlens, const int32_t* prefi
       for (int j = 0; j <= i; ++j) {
         int c = psa::classify(i, j, len, cs, rs, false);
         if (!c) continue;
-        p->fwd_entries.push_back((j << 1) | (c == 2));
+        p->fwd_entries.push_back((j << 2) | (int(psa::precise_rows(i, len, cs, rs)) << 1) | (c == 2));
         ++r.list_cnt;
         ++p->live_tiles;
         p->partial_tiles += (c == 2);
@@ -123,7 +133,7 @@ extern "C" psa_status_t psa_plan(const int32_t* cu_seqlens, const int32_t* prefi
       for (int i = j; i < nt; ++i) {
         int c = psa::classify(i, j, len, cs, rs, true);
         if (!c) continue;
-        p->bwd_entries.push_back((i << 1) | (c == 2));
+        p->bwd_entries.push_back((i << 2) | (int(psa::precise_rows(i, len, cs, rs)) << 1) | (c == 2));
         ++r.list_cnt;
       }
       p->kv_tiles.push_back(r);

@@ -53,6 +53,7 @@ def _check_against_dense_mask(pack):
         return 1 if full else 2
 
     fwd_set, n_live, n_partial = {}, 0, 0
+    precise_of = {}
     seen_tiles = set()
     for row0, ds, local0, length, cs, rs, off, cnt in f_tiles:
         s = sample_of[int(ds)]
@@ -60,9 +61,14 @@ def _check_against_dense_mask(pack):
         assert row0 == ds + local0 and local0 % TILE == 0 and local0 < length
         i = local0 // TILE
         seen_tiles.add((s, i))
-        listed = {int(e) >> 1: int(e) & 1 for e in f_ent[off:off + cnt]}
+        listed = {int(e) >> 2: int(e) & 1 for e in f_ent[off:off + cnt]}
+        precise = {int(e) >> 2: (int(e) >> 1) & 1 for e in f_ent[off:off + cnt]}
         assert len(listed) == cnt
-        assert sorted(listed) == [int(e) >> 1 for e in f_ent[off:off + cnt]], "key tiles must ascend"
+        assert sorted(listed) == [int(e) >> 2 for e in f_ent[off:off + cnt]], "key tiles must ascend"
+        q_lo, q_hi = int(ds) + i * TILE, min(int(ds) + i * TILE + TILE, int(ds) + int(length))
+        few_keys = bool((mask[q_lo:q_hi].sum(axis=1) < TILE).any())
+        assert all(p == int(few_keys) for p in precise.values()), (s, i, few_keys)
+        precise_of[(s, i)] = int(few_keys)
         for j in range((length + TILE - 1) // TILE):
             c = dense_class(int(ds), int(length), i, j, False)
             if c == 0:
@@ -87,12 +93,13 @@ def _check_against_dense_mask(pack):
         s = sample_of[int(ds)]
         j = local0 // TILE
         for e in b_ent[off:off + cnt]:
-            i = int(e) >> 1
+            i = int(e) >> 2
             c = dense_class(int(ds), int(length), i, j, True)
             assert c != 0
             if c == 2:
                 assert int(e) & 1 == 1, (s, i, j)
             bwd_set[(s, i, j)] = int(e) & 1
+            assert (int(e) >> 1) & 1 == precise_of[(s, i)], (s, i, j)
     assert set(bwd_set) == set(fwd_set), "forward and transposed maps hold the same tiles"
     plan.close()
 
