@@ -158,6 +158,41 @@ psa_status_t psa_bwd(const psa_plan_t* plan, const void* d_o, const void* q, con
                      int32_t* device_status, void* stream);
 
 /*
+ * psa_bwd_static_scratch -- psa_bwd without the workspace argument.  The paper has no
+ * counterpart; this entry point exists for callers that have no way to provide scratch
+ * memory at the time of the call: for example a step function running after the
+ * framework's caching allocator has taken the whole device (a raw cudaMalloc from a
+ * library would fail or fragment it), or a latency-critical loop that must not trigger
+ * the device-wide synchronisation that cudaMalloc / cudaFree imply.
+ *
+ * The call allocates nothing: no cudaMalloc, no cudaFree, no allocating library routine.
+ * Its scratch (the fp32 dq accumulator and the delta vector) is a fixed array of
+ * PSA_STATIC_SCRATCH_BYTES (32 MiB) inside the library's device image; every GPU that
+ * loads the library holds that array until the process exits.
+ *
+ *   Arguments   as psa_bwd, minus `workspace`.  Inputs and outputs are still the caller's.
+ *   Limit       plans with psa_plan_stats().bwd_workspace_bytes > PSA_STATIC_SCRATCH_BYTES
+ *               (roughly T * Hq * d > 8.3 M elements, e.g. more than 2030 tokens at 32
+ *               heads of 128) are rejected with PSA_ERR_UNSUPPORTED before anything is
+ *               launched; with PSA_DEBUG set in the environment the sizes are printed.
+ *   First call  the first call on each device looks up the array's device address (with
+ *               that device current) and keeps it.  Make that first call before any stream
+ *               capture begins on the device.
+ *   Sharing     all calls on a device use the same array, which keeps the previous call's
+ *               contents.  The call itself clears the part that must start at zero (the dq
+ *               accumulator) and overwrites the rest before reading it, so calls that run
+ *               one after another are independent.  Two calls that overlap on the GPU
+ *               (different streams, or different host threads) race on the array and give
+ *               wrong gradients: serialise them.
+ * Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED (too large), CUDA.
+ */
+#define PSA_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+psa_status_t psa_bwd_static_scratch(const psa_plan_t* plan, const void* d_o, const void* q,
+                                    const void* k, const void* v, const void* o, const float* lse,
+                                    void* dq, void* dk, void* dv, int32_t* device_status,
+                                    void* stream);
+
+/*
  * dpo_logp -- summed log-probabilities per response (Section 2.1: the total
  * log probability of each completion; Section 3.2: responses are recovered at
  * loss time from their boundaries).

@@ -17,12 +17,14 @@ _LIB_PATH = os.path.join(_HERE, "libpsa.so")
 _lib = None
 
 PSA_PLAN_HOST_ONLY = 1
+PSA_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 PSA_DTYPE_F32, PSA_DTYPE_BF16 = 0, 1
 PSA_DEVSTAT_WAIT_EXPIRED, PSA_DEVSTAT_BAD_TARGET, PSA_DEVSTAT_BAD_SEGMENT = 1, 2, 4
 
 EXPORTED_SYMBOLS = (
     "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
     "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp", "psa_profile_events",
+    "psa_bwd_static_scratch",
 )
 
 
@@ -59,6 +61,7 @@ def load_library():
     lib.psa_plan_export.argtypes = [vp, i32, vp, vp]
     lib.psa_fwd.argtypes = [vp] * 8
     lib.psa_bwd.argtypes = [vp] * 13
+    lib.psa_bwd_static_scratch.argtypes = [vp] * 12
     lib.psa_profile_events.argtypes = [i32, vp, vp]
     lib.dpo_logp.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     for name in EXPORTED_SYMBOLS:
@@ -215,3 +218,19 @@ def psa_profile_events(which, start=None, stop=None):
     a = C.c_void_p(0) if start is None else C.c_void_p(start.cuda_event)
     b = C.c_void_p(0) if stop is None else C.c_void_p(stop.cuda_event)
     _check("psa_profile_events", load_library().psa_profile_events(which, a, b))
+
+
+def psa_bwd_static_scratch(plan: Plan, d_o, q, k, v, o, lse, dq, dk, dv, status=None, stream=None):
+    """psa_bwd for callers that cannot provide a workspace (for instance because all device
+    memory already belongs to the framework's allocator): the scratch is a fixed 32 MiB
+    array inside the library.  Nothing is allocated here either: the three gradient tensors
+    must be passed in.  Plans whose scratch need exceeds PSA_STATIC_SCRATCH_BYTES raise
+    PsaError (status 3).  Calls that overlap on the GPU share the array and must be serialised."""
+    import torch
+    for t in (d_o, q, k, v, o, dq, dk, dv):
+        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    assert lse.dtype == torch.float32 and lse.is_contiguous()
+    _check("psa_bwd_static_scratch",
+           load_library().psa_bwd_static_scratch(plan._h, _ptr(d_o), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
+                                                 _ptr(dq), _ptr(dk), _ptr(dv), _ptr(status), _stream(stream)))
+    return dq, dk, dv
