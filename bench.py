@@ -84,6 +84,22 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
+def max_over_ranks(values, device):
+    """Element-wise maximum of a list of floats over all ranks (identity on one rank).
+    The path has no exchange step: this reduction of the timings is the only collective."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_tflops(flops_per_replica, world, ms):
+    """N independent replicas: the job's work is the sum, its time the slowest rank's."""
+    return world * flops_per_replica / ms / 1e9
+
+
 def oracle_sample(pack, steps, warmup, target="bench"):
     """Times the fp64 oracle, as it stands, on a bounded sample of the workload:
     whole samples of the pack (attention is independent per sample) and one kv
@@ -285,17 +301,15 @@ def main():
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     # ---- max over ranks (replicas): whole-job value = sum of the replicas' useful flops / slowest time
-    times = torch.tensor([step_ms, att_ms, lp_ms, e2e["ms_per_step"] if e2e else 0.0], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    step_ms, att_ms, lp_ms, e2e_ms_max = (float(x) for x in times.cpu())
+    step_ms, att_ms, lp_ms, e2e_ms_max = max_over_ranks(
+        [step_ms, att_ms, lp_ms, e2e["ms_per_step"] if e2e else 0.0], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     peaks = measured_peaks()
-    value = world * (flops_fwd + flops_bwd) / att_ms / 1e9
+    value = whole_job_tflops(flops_fwd + flops_bwd, world, att_ms)
     bwd_ms, fwd_ms, klp_ms = (float(np.mean(kernel_ms[n])) for n in ("bwd", "fwd", "logp"))
     bwd_tflops = flops_bwd / bwd_ms / 1e9
     logp_bytes = live_rows * VOCAB * 2 + 8 * live_rows + 4 * n_seg
@@ -328,7 +342,7 @@ def main():
         "paper_context": "paper reports 1.1-1.5x (1.3-1.6x with packing) end-to-end training speedups on 8xH100; context, not the target",
     }
     if e2e:
-        e2e["value"] = world * (flops_fwd + flops_bwd) / e2e_ms_max / 1e9
+        e2e["value"] = whole_job_tflops(flops_fwd + flops_bwd, world, e2e_ms_max)
         e2e["ms_per_step"] = e2e_ms_max
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
