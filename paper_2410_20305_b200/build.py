@@ -27,6 +27,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+    if os.environ.get("PSA_EXPERIMENT"):   # timing experiments, results invalid
+        cmd += ["-D" + os.environ["PSA_EXPERIMENT"]]
+    if os.environ.get("PSA_TRACE"):   # debug build: hand-off timestamps of the backward kernel
+        cmd += ["-DPSA_TRACE"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     res = subprocess.run(cmd, capture_output=True, text=True)

@@ -12,12 +12,15 @@
 //          dV  += P^T dO         dK  += dS^T Q          dQ_i = dS K  (added into dq_accum)
 //   3. convert:     dq = bf16(dq_accum)
 //
-// Warp roles of the main kernel (320 threads, one CTA per SM):
-//   warp 0      TMA producer: K, V once; Q and dO double-buffered per iteration
-//   warp 1      UMMA issuer (tcgen05, all five products)
-//   warps 2..5  compute: one thread per key row; P^T -> TMEM (bf16, over S^T),
-//               dS^T -> shared memory (bf16, 128-byte swizzle) for the dK and dQ products
-//   warps 6..9  dQ drain: TMEM -> registers -> vector red.add into the fp32 dq_accum
+// Warp roles of the main kernel (512 threads = 4 warpgroups, one CTA per SM):
+//   warp 0        TMA producer: K, V once; Q double-buffered, dO single-buffered per iteration
+//   warp 1        UMMA issuer (tcgen05, all five products); warps 2, 3 idle
+//   warps 4..11   workers: one thread per (key row, half of the 128 query columns);
+//                 P^T -> TMEM (bf16, over S^T), dS^T -> shared memory (bf16, 128-byte swizzle) for
+//                 the dK and dQ products
+//   warps 12..15  dQ drain: TMEM -> registers (columns released at once) -> shared-memory staging
+//                 -> TMA reduce-add (cp.reduce.async.bulk.tensor, fp32) into dq_accum
+// Registers are moved between the warpgroups with setmaxnreg (the drain holds a whole dQ row).
 // TMEM columns: [0,128) S^T / P^T, [128,256) dP^T / dQ, [256,256+D) dV, [384,384+D) dK.
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -30,11 +33,14 @@
 #include "psa_tensormap.h"
 
 namespace psa {
+#ifdef PSA_TRACE
+__device__ long long g_psa_trace[64 * 16];
+#endif
 namespace {
 
 using namespace dev;
 
-constexpr int kBwdThreads = 320;
+constexpr int kBwdThreads = 512;   // 16 warps = 4 warpgroups, see the role table above
 constexpr uint32_t kBwdTmemCols = 512;
 constexpr uint32_t kColS = 0, kColDP = 128, kColDV = 256, kColDK = 384;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -42,6 +48,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 struct BwdParams {
   const TileRec* tiles;     // key tiles
   const int32_t* entries;   // (query tile << 2) | (precise << 1) | needs_mask
+  const int32_t* cta_map;   // per CTA: (key tile record, kv head)
   const float* lse;         // [Hq, T]
   const float* delta;       // [Hq, T]
   float* dq_accum;          // [T, Hq, D] fp32
@@ -58,22 +65,37 @@ struct BwdSmem {
   static constexpr int kTileBytes = kTile * D * 2;      // K, V, Q, dO tiles
   static constexpr int kSubBytes = kTile * 128;
   static constexpr int kDsBytes = kTile * kTile * 2;    // dS^T tile, 128 x 128 bf16
-  static constexpr int kK = 0, kV = kTileBytes, kQ = 2 * kTileBytes, kDO = 4 * kTileBytes, kDS = 6 * kTileBytes;
+  static constexpr int kStageBytes = kTile * 32 * 4;    // dQ staging: 128 rows x 32 fp32 columns
+  static constexpr int kK = 0, kV = kTileBytes, kQ = 2 * kTileBytes /* 2 stages */, kDO = 4 * kTileBytes;
+  static constexpr int kDQS = 5 * kTileBytes;           // 2 staging buffers
+  static constexpr int kDS = kDQS + 2 * kStageBytes;
   static constexpr int kBars = kDS + kDsBytes;          // 16 mbarriers
   static constexpr int kTmemSlot = kBars + 128;
   static constexpr int kAbort = kTmemSlot + 4;
   static constexpr int kLse = kBars + 256;              // [2][128] floats
   static constexpr int kDelta = kLse + 1024;            // [2][128] floats
-  static constexpr int kBytes = kDelta + 1024;
+  static constexpr int kEnt = kDelta + 1024;            // first kEntCap entries of the tile's list
+  static constexpr int kEntCap = 128;
+  static constexpr int kBytes = kEnt + kEntCap * 4;
   // More than half an SM's shared memory: exactly one CTA per SM, so the
   // 512-column TMEM allocation never has to wait for a neighbour.
   static constexpr int kRequest = kBytes > 120 * 1024 ? kBytes : 120 * 1024;
 };
 
 enum {
-  B_KV_FULL = 0, B_Q_FULL0, B_Q_FULL1, B_DO_FULL0, B_DO_FULL1, B_QDO_EMPTY0, B_QDO_EMPTY1,
-  B_S_FULL, B_DP_FULL, B_P_FULL, B_DS_FULL, B_DS_EMPTY, B_DQ_FULL, B_DQ_EMPTY, B_COUNT
+  B_KV_FULL = 0, B_Q_FULL0, B_Q_FULL1, B_Q_EMPTY0, B_Q_EMPTY1, B_DO_FULL, B_DO_EMPTY,
+  B_S_FULL, B_DP_FULL, B_P_FULL, B_DS_FULL, B_DS_EMPTY, B_DQ_FULL, B_DQ_EMPTY, B_DONE, B_COUNT
 };
+
+// Debug builds (-DPSA_TRACE) record SM-clock timestamps of the first CTA's hand-offs.
+#ifdef PSA_TRACE
+#define PSA_TRACE_MARK(it, slot)                                                        \
+  do {                                                                                  \
+    if (blockIdx.x == 0 && (it) < 64) g_psa_trace[(it) * 16 + (slot)] = clock64();       \
+  } while (0)
+#else
+#define PSA_TRACE_MARK(it, slot) do {} while (0)
+#endif
 
 __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
@@ -89,13 +111,14 @@ template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-               const BwdParams prm) {
+               const __grid_constant__ CUtensorMap tm_dq, const BwdParams prm) {
   using L = BwdSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
   const uint32_t sK = base + L::kK, sV = base + L::kV, sDS = base + L::kDS;
   auto sQ = [&](int st) { return base + L::kQ + st * L::kTileBytes; };
-  auto sDO = [&](int st) { return base + L::kDO + st * L::kTileBytes; };
+  const uint32_t sDO = base + L::kDO;
+  int32_t* s_ent = reinterpret_cast<int32_t*>(smem_raw + L::kEnt);
   auto bar = [&](int i) { return base + L::kBars + 8u * i; };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + L::kTmemSlot);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + L::kAbort);
@@ -103,8 +126,8 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   float* s_delta = reinterpret_cast<float*>(smem_raw + L::kDelta);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile_idx = blockIdx.x / prm.Hkv;
-  const int hk = blockIdx.x % prm.Hkv;
+  const int tile_idx = prm.cta_map[2 * blockIdx.x];
+  const int hk = prm.cta_map[2 * blockIdx.x + 1];
   const int g = prm.Hq / prm.Hkv;
   const TileRec rec = prm.tiles[tile_idx];
   const int32_t* ent = prm.entries + rec.list_off;
@@ -120,11 +143,12 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (prm.status) atomicOr(prm.status, PSA_DEVSTAT_WAIT_EXPIRED);
     }
     for (int i = 0; i < B_COUNT; ++i) {
-      const bool many = (i == B_P_FULL || i == B_DS_FULL || i == B_DQ_EMPTY);
-      mbar_init(bar(i), many ? 128 : 1);
+      mbar_init(bar(i), (i == B_P_FULL || i == B_DS_FULL) ? 256 : (i == B_DQ_EMPTY ? 128 : 1));
     }
     fence_mbar_init();
   }
+  // The list is read by every role in every iteration: keep its head in shared memory.
+  if (int(threadIdx.x) < n_list && int(threadIdx.x) < L::kEntCap) s_ent[threadIdx.x] = ent[threadIdx.x];
   if (warp == 0) tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kBwdTmemCols);
   tc_fence_before();
   __syncthreads();
@@ -133,8 +157,15 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
   // Iteration it -> (query head of the group, entry of the list).
   auto head_of = [&](int it) { return hk * g + it / n_list; };
-  auto entry_of = [&](int it) { return ent[it % n_list]; };
+  auto entry_of = [&](int it) {
+    const int li = it % n_list;
+    return li < L::kEntCap ? s_ent[li] : ent[li];
+  };
 
+  // Each warpgroup changes its register budget as its first action, inside its own branch, so
+  // that everything the branch executes afterwards is compiled for that budget.
+  if (warp < 4) {
+  setmaxnreg_dec<72>();
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -142,6 +173,7 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       tma_prefetch_desc(&tm_k);
       tma_prefetch_desc(&tm_v);
       tma_prefetch_desc(&tm_do);
+      tma_prefetch_desc(&tm_dq);
       mbar_expect_tx(bar(B_KV_FULL), 2 * L::kTileBytes);
       for (int s = 0; s < L::kSub; ++s) tma_load_3d(sK + s * L::kSubBytes, &tm_k, s * 64, hk, rec.row0, bar(B_KV_FULL));
       for (int s = 0; s < L::kSub; ++s) tma_load_3d(sV + s * L::kSubBytes, &tm_v, s * 64, hk, rec.row0, bar(B_KV_FULL));
@@ -149,11 +181,13 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int st = it & 1;
         const int h = head_of(it);
         const int qrow = rec.ds + (entry_of(it) >> 2) * kTile;
-        if (it >= 2) mbar_wait(bar(B_QDO_EMPTY0 + st), ((it >> 1) - 1) & 1, wctx);
+        if (it >= 2) mbar_wait(bar(B_Q_EMPTY0 + st), ((it >> 1) - 1) & 1, wctx);
         mbar_expect_tx(bar(B_Q_FULL0 + st), L::kTileBytes);
         for (int s = 0; s < L::kSub; ++s) tma_load_3d(sQ(st) + s * L::kSubBytes, &tm_q, s * 64, h, qrow, bar(B_Q_FULL0 + st));
-        mbar_expect_tx(bar(B_DO_FULL0 + st), L::kTileBytes);
-        for (int s = 0; s < L::kSub; ++s) tma_load_3d(sDO(st) + s * L::kSubBytes, &tm_do, s * 64, h, qrow, bar(B_DO_FULL0 + st));
+        if (it >= 1) mbar_wait(bar(B_DO_EMPTY), (it - 1) & 1, wctx);   // dV of the previous iteration has read dO
+        PSA_TRACE_MARK(it, 11);
+        mbar_expect_tx(bar(B_DO_FULL), L::kTileBytes);
+        for (int s = 0; s < L::kSub; ++s) tma_load_3d(sDO + s * L::kSubBytes, &tm_do, s * 64, h, qrow, bar(B_DO_FULL));
       }
     }
     __syncwarp();
@@ -164,95 +198,127 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       constexpr uint32_t idesc_dv = umma_idesc_bf16(kTile, D, false, true);       // P^T (TMEM) x dO (MN-major)
       constexpr uint32_t idesc_dk = umma_idesc_bf16(kTile, D, false, true);       // dS^T (K-major) x Q (MN-major)
       constexpr uint32_t idesc_dq = umma_idesc_bf16(kTile, D, true, true);        // dS (MN-major) x K (MN-major)
+      // Low descriptor words of every operand view (K-major: _k, MN-major: _mn); a K step of 16
+      // elements advances a K-major operand by 32 bytes inside its 64-element sub-tile and an
+      // MN-major operand by 16 rows (2048 bytes).
+      const uint32_t k_k = smem_desc_lo(sK, 16), v_k = smem_desc_lo(sV, 16), do_k = smem_desc_lo(sDO, 16);
+      const uint32_t q0_k = smem_desc_lo(sQ(0), 16), q1_k = smem_desc_lo(sQ(1), 16);
+      const uint32_t ds_k = smem_desc_lo(sDS, 16), ds_mn = smem_desc_lo(sDS, 16384);
+      const uint32_t do_mn = smem_desc_lo(sDO, L::kSubBytes), k_mn = smem_desc_lo(sK, L::kSubBytes);
+      const uint32_t q0_mn = smem_desc_lo(sQ(0), L::kSubBytes), q1_mn = smem_desc_lo(sQ(1), L::kSubBytes);
       mbar_wait(bar(B_KV_FULL), 0, wctx);
       uint32_t ds_ph = 0;  // running parity of B_DS_FULL (it completes twice in a PRECISE iteration)
-      for (int it = 0; it < n_it; ++it) {
+      // S^T = K Q^T of iteration `it`.  Its columns hold P^T of the previous iteration; the dV
+      // product that reads it is always issued earlier by this thread and UMMAs execute in issue order.
+      auto issue_s = [&](int it) {
         const int st = it & 1, ph = (it >> 1) & 1;
-        // PRECISE tiles carry P^T and dS^T as two bf16 terms each.
-        const int n_terms = (entry_of(it) & 2) ? 2 : 1;
-        // S^T = K Q^T.  (Its columns held P^T of the previous iteration; the dV product that
-        // read it was issued earlier by this thread and UMMAs execute in issue order.)
         mbar_wait(bar(B_Q_FULL0 + st), ph, wctx);
         tc_fence_after();
+        PSA_TRACE_MARK(it, 0);
+        const uint32_t q_lo = st ? q1_k : q0_k;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * L::kSubBytes + (kk & 3) * 32;
-          umma_ss(tmem + kColS, smem_desc_sw128(sK + off, 16, 1024), smem_desc_sw128(sQ(st) + off, 16, 1024), idesc_st,
-                  kk > 0);
+          const uint32_t off = ((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4;
+          umma_ss_lo(tmem + kColS, k_k + off, q_lo + off, idesc_st, kk > 0);
         }
         umma_commit(bar(B_S_FULL));
-        // dP^T = V dO^T into the columns the previous dQ occupied: wait until it was drained.
-        mbar_wait(bar(B_DO_FULL0 + st), ph, wctx);
+      };
+      issue_s(0);
+      for (int it = 0; it < n_it; ++it) {
+        const int st = it & 1;
+        // PRECISE tiles carry P^T and dS^T as two bf16 terms each.
+        const int n_terms = (entry_of(it) & 2) ? 2 : 1;
+        // dP^T = V dO^T into the columns the previous dQ occupied: wait until it was read out.
+        // (This commit also covers the previous iteration's dK / dQ products, so a completed
+        // dP^T tells the compute warps that the dS buffer is free again.)
+        PSA_TRACE_MARK(it, 13);
+        mbar_wait(bar(B_DO_FULL), it & 1, wctx);
+        PSA_TRACE_MARK(it, 14);
         if (it > 0) mbar_wait(bar(B_DQ_EMPTY), (it - 1) & 1, wctx);
         tc_fence_after();
+        PSA_TRACE_MARK(it, 1);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * L::kSubBytes + (kk & 3) * 32;
-          umma_ss(tmem + kColDP, smem_desc_sw128(sV + off, 16, 1024), smem_desc_sw128(sDO(st) + off, 16, 1024),
-                  idesc_st, kk > 0);
+          const uint32_t off = ((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4;
+          umma_ss_lo(tmem + kColDP, v_k + off, do_k + off, idesc_st, kk > 0);
         }
         umma_commit(bar(B_DP_FULL));
         // dV += P^T dO   (reduction over the 128 query rows, 16 per instruction)
         mbar_wait(bar(B_P_FULL), it & 1, wctx);
         tc_fence_after();
-        for (int term = 0; term < n_terms; ++term) {   // second term: columns [64,128) of the S region
+        PSA_TRACE_MARK(it, 2);
+        // P^T of query columns [64 h, 64 h + 64) sits in S-region columns [64 h, 64 h + 32), the
+        // second term of a PRECISE tile in [64 h + 32, 64 h + 64); 16 queries = 8 columns.
+        for (int term = 0; term < n_terms; ++term) {
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk)
-            umma_ts(tmem + kColDV, tmem + kColS + term * 64 + kk * 8,
-                    smem_desc_sw128(sDO(st) + kk * 2048, L::kSubBytes, 1024), idesc_dv,
-                    (it > 0) || (kk > 0) || (term > 0));
+            umma_ts_lo(tmem + kColDV, tmem + kColS + (kk >> 2) * 64 + term * 32 + (kk & 3) * 8,
+                       do_mn + kk * (2048 >> 4), idesc_dv, (it > 0) || (kk > 0) || (term > 0));
         }
+        umma_commit(bar(B_DO_EMPTY));
+        PSA_TRACE_MARK(it, 15);
+        // The next S^T goes in now, so that the compute warps can start on it while the dK / dQ
+        // products of this iteration run.
+        if (it + 1 < n_it) issue_s(it + 1);
         // dK += dS^T Q ; dQ = dS K.  The two terms of a PRECISE tile pass through the one
         // shared-memory buffer one after the other.
         for (int term = 0; term < n_terms; ++term) {
           mbar_wait(bar(B_DS_FULL), ds_ph, wctx);
           ds_ph ^= 1;
           tc_fence_after();
+          PSA_TRACE_MARK(it, 3);
+          // dQ first: the workers are waiting to read it out, and the next dP^T for them to finish.
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk)
-            umma_ss(tmem + kColDK, smem_desc_sw128(sDS + (kk >> 2) * 16384 + (kk & 3) * 32, 16, 1024),
-                    smem_desc_sw128(sQ(st) + kk * 2048, L::kSubBytes, 1024), idesc_dk,
-                    (it > 0) || (kk > 0) || (term > 0));
+            umma_ss_lo(tmem + kColDP, ds_mn + kk * (2048 >> 4), k_mn + kk * (2048 >> 4), idesc_dq,
+                       (kk > 0) || (term > 0));
+          if (term + 1 == n_terms) umma_commit(bar(B_DQ_FULL));
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk)
-            umma_ss(tmem + kColDP, smem_desc_sw128(sDS + kk * 2048, 16384, 1024),
-                    smem_desc_sw128(sK + kk * 2048, L::kSubBytes, 1024), idesc_dq, (kk > 0) || (term > 0));
+            umma_ss_lo(tmem + kColDK, ds_k + (((kk >> 2) * 16384 + (kk & 3) * 32) >> 4),
+                       (st ? q1_mn : q0_mn) + kk * (2048 >> 4), idesc_dk, (it > 0) || (kk > 0) || (term > 0));
           if (term + 1 < n_terms) umma_commit(bar(B_DS_EMPTY));
         }
-        umma_commit(bar(B_DQ_FULL));
-        umma_commit(bar(B_QDO_EMPTY0 + st));
+        umma_commit(bar(B_Q_EMPTY0 + st));
+        PSA_TRACE_MARK(it, 4);
       }
+      umma_commit(bar(B_DONE));   // every product, the last dK included, has completed
     }
     __syncwarp();
-  } else if (warp < 6) {
-    // ------------------------------------------------------------ compute, one key row per thread
+  }  // warps 2, 3 of the first warpgroup are idle
+  } else if (warp < 12) {
+    // ------------------------------------------------------------ workers: warps 4..11
+    // Thread = one key row (TMEM lane) and one half of the 128 query columns: warps 4..7 take
+    // columns [0,64), warps 8..11 columns [64,128).
+    setmaxnreg_inc<144>();
+    constexpr int DH = D / 2;                           // dV / dK columns per worker in the epilogue
     const int quarter = warp & 3;
+    const int half = (warp - 4) >> 2;
     const int r = quarter * 32 + lane;
     const uint32_t lane_base = uint32_t(quarter * 32) << 16;
-    const int ct = threadIdx.x - 64;                    // 0..127 among the compute threads
+    const int wt = threadIdx.x - 128;                   // 0..255 among the workers
+    const int c0 = half * 64;                           // first query column of this thread
+    const bool leader = wt == 0;
     const int kv_local = rec.local0 + r;
     const bool kv_valid = kv_local < rec.len;
     // Queries allowed to see this key: [kv_local, qend).
     const int qend = (kv_local >= rec.cs && kv_local < rec.rs) ? rec.rs : rec.len;
     const float cl = prm.scale_log2;
 
-    auto load_stats = [&](int it, float& l2, float& dl) {
-      const int64_t qrow = int64_t(rec.ds) + (entry_of(it) >> 2) * kTile + ct;
-      l2 = 0.f;
-      dl = 0.f;
+    // Per-column statistics of the iteration's query tile: workers 0..127 fetch lse * log2e,
+    // workers 128..255 fetch delta, each for column (wt & 127).
+    auto load_stat = [&](int it) {
+      const int64_t qrow = int64_t(rec.ds) + (entry_of(it) >> 2) * kTile + (wt & 127);
+      float x = 0.f;
       if (qrow < prm.T) {
         const int64_t idx = int64_t(head_of(it)) * prm.T + qrow;
-        l2 = prm.lse[idx] * kLog2e;
-        dl = prm.delta[idx];
+        x = wt < 128 ? prm.lse[idx] * kLog2e : prm.delta[idx];
       }
+      return x;
     };
-    {
-      float l2, dl;
-      load_stats(0, l2, dl);
-      s_lse[ct] = l2;
-      s_delta[ct] = dl;
-    }
-    named_bar_sync(1, 128);
+    auto store_stat = [&](int st, float x) { (wt < 128 ? s_lse : s_delta)[st * kTile + (wt & 127)] = x; };
+    store_stat(0, load_stat(0));
+    named_bar_sync(1, 256);
 
     uint32_t dse_ph = 0;  // running parity of B_DS_EMPTY
 
@@ -264,74 +330,73 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int st = it & 1;
       const int e = entry_of(it);
       const int q0 = (e >> 2) * kTile;
-      float nl2 = 0.f, ndl = 0.f;
-      if (it + 1 < n_it) load_stats(it + 1, nl2, ndl);
+      float next_stat = 0.f;
+      if (it + 1 < n_it) next_stat = load_stat(it + 1);
 
       mbar_wait(bar(B_S_FULL), it & 1, wctx);
       tc_fence_after();
-      float p[kTile];
-#pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t v[32];
-        tmem_ld32(tmem + lane_base + kColS + ch * 32, v);
-        tc_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) p[ch * 32 + i] = __uint_as_float(v[i]);
-      }
+      if (leader) PSA_TRACE_MARK(it, 5);
+      float p[64];
       {
-        const float4* l4 = reinterpret_cast<const float4*>(s_lse + st * kTile);
+        uint32_t sv[64];   // both loads in flight, one wait
+        tmem_ld64_wait(tmem + lane_base + kColS + c0, sv);
+        if (leader) PSA_TRACE_MARK(it, 12);
+        const float4* l4 = reinterpret_cast<const float4*>(s_lse + st * kTile + c0);
 #pragma unroll
-        for (int i = 0; i < kTile / 4; ++i) {
+        for (int i = 0; i < 16; ++i) {
           const float4 l = l4[i];
-          p[4 * i + 0] = ex2_approx(fmaf(p[4 * i + 0], cl, -l.x));
-          p[4 * i + 1] = ex2_approx(fmaf(p[4 * i + 1], cl, -l.y));
-          p[4 * i + 2] = ex2_approx(fmaf(p[4 * i + 2], cl, -l.z));
-          p[4 * i + 3] = ex2_approx(fmaf(p[4 * i + 3], cl, -l.w));
+          p[4 * i + 0] = ex2_approx(fmaf(__uint_as_float(sv[4 * i + 0]), cl, -l.x));
+          p[4 * i + 1] = ex2_approx(fmaf(__uint_as_float(sv[4 * i + 1]), cl, -l.y));
+          p[4 * i + 2] = ex2_approx(fmaf(__uint_as_float(sv[4 * i + 2]), cl, -l.z));
+          p[4 * i + 3] = ex2_approx(fmaf(__uint_as_float(sv[4 * i + 3]), cl, -l.w));
         }
       }
       if (e & 1) {
-        const int lo = kv_local - q0;                        // first allowed column (causal)
-        const int hi = qend - q0;                            // one past the last allowed column
+        const int lo = kv_local - q0 - c0;                   // first allowed column (causal), relative to c0
+        const int hi = qend - q0 - c0;                       // one past the last allowed column
         const uint32_t span = hi > lo ? uint32_t(hi - lo) : 0u;
 #pragma unroll
-        for (int i = 0; i < kTile; ++i) p[i] = (uint32_t(i - lo) < span) ? p[i] : 0.f;
+        for (int i = 0; i < 64; ++i) p[i] = (uint32_t(i - lo) < span) ? p[i] : 0.f;
       }
-#pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
+      {
+        // bf16 pairs: this half's 64 probabilities go to the first 32 of the 64 S^T columns this
+        // thread has just read (never into the other half's columns: the thread of the other
+        // half may not have read its S^T yet); the second term of a PRECISE tile to the last 32.
         uint32_t v[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = pack_bf16x2(p[ch * 64 + 2 * i], p[ch * 64 + 2 * i + 1]);
-        tmem_st32(tmem + lane_base + kColS + ch * 32, v);
+        for (int i = 0; i < 32; ++i) v[i] = pack_bf16x2(p[2 * i], p[2 * i + 1]);
+        tmem_st32(tmem + lane_base + kColS + half * 64, v);
         if constexpr (kPrecise) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = pack_bf16x2_residual(p[ch * 64 + 2 * i], p[ch * 64 + 2 * i + 1], v[i]);
-          tmem_st32(tmem + lane_base + kColS + 64 + ch * 32, v);
+          for (int i = 0; i < 32; ++i) v[i] = pack_bf16x2_residual(p[2 * i], p[2 * i + 1], v[i]);
+          tmem_st32(tmem + lane_base + kColS + half * 64 + 32, v);
         }
       }
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar(B_P_FULL));
+      if (leader) PSA_TRACE_MARK(it, 6);
 
-      // dS^T = P^T * (dP^T - delta) -> shared memory.  The buffer is free: S^T of this
-      // iteration completed after the previous iteration's dK / dQ products.
+      // dS^T = P^T * (dP^T - delta) -> shared memory.  The buffer is free: dP^T of this
+      // iteration was issued, and so completed, after the previous iteration's dK / dQ products.
       mbar_wait(bar(B_DP_FULL), it & 1, wctx);
       tc_fence_after();
+      if (leader) PSA_TRACE_MARK(it, 7);
       if constexpr (kPrecise) {
         if ((e >> 2) == 0) {
           // Rows of a sample's first query tile see only this key tile, and they are the rows
           // with few keys, where delta = dO . O computed from the bf16-rounded O is the largest
           // error left.  Recompute it exactly here:  delta_i = sum_j P_ij dP_ij  (fp32).
           // Column sums over the 128 key rows: transpose-reduce inside each warp, then add the
-          // four warps through the (still unused) dS buffer.
+          // four warps of each half through the (still unused) dS buffer.
           float* scratch = reinterpret_cast<float*>(smem_raw + L::kDS);
 #pragma unroll
-          for (int ch = 0; ch < 4; ++ch) {
+          for (int j = 0; j < 2; ++j) {
             uint32_t v[32];
-            tmem_ld32(tmem + lane_base + kColDP + ch * 32, v);
-            tc_wait_ld();
+            tmem_ld32_wait(tmem + lane_base + kColDP + c0 + j * 32, v);
             float t[32];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) t[i] = p[ch * 32 + i] * __uint_as_float(v[i]);
+            for (int i = 0; i < 32; ++i) t[i] = p[j * 32 + i] * __uint_as_float(v[i]);
 #pragma unroll
             for (int off = 16; off >= 1; off >>= 1) {
               const bool up = (lane & off) != 0;
@@ -342,90 +407,87 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                 t[kq] = keep + __shfl_xor_sync(0xffffffffu, send, off);
               }
             }
-            scratch[quarter * kTile + ch * 32 + lane] = t[0];   // lane l now holds column ch*32 + l
+            scratch[quarter * kTile + c0 + j * 32 + lane] = t[0];   // lane l holds column c0 + 32 j + l
           }
-          named_bar_sync(1, 128);
-          const float dsum = scratch[ct] + scratch[kTile + ct] + scratch[2 * kTile + ct] + scratch[3 * kTile + ct];
-          s_delta[st * kTile + ct] = dsum;
-          named_bar_sync(1, 128);
+          named_bar_sync(1, 256);
+          if (wt < kTile)
+            s_delta[st * kTile + wt] = scratch[wt] + scratch[kTile + wt] + scratch[2 * kTile + wt] + scratch[3 * kTile + wt];
+          named_bar_sync(1, 256);
         }
       }
-      const float4* d4 = reinterpret_cast<const float4*>(s_delta + st * kTile);
-      uint32_t ds_lo[kPrecise ? 64 : 1];  // second bf16 term of dS^T
+      const float4* d4 = reinterpret_cast<const float4*>(s_delta + st * kTile + c0);
+      uint32_t ds_lo[kPrecise ? 32 : 1];  // second bf16 term of dS^T
+      // Row r of this half's 128 x 64 bf16 sub-tile: eight 16-byte chunks, each stored at chunk
+      // index XOR (r & 7)  (128-byte swizzle).
+      const uint32_t row_addr = sDS + half * 16384 + r * 128;
 #pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
+      for (int j = 0; j < 2; ++j) {
         uint32_t v[32];
-        tmem_ld32(tmem + lane_base + kColDP + ch * 32, v);
-        tc_wait_ld();
+        tmem_ld32_wait(tmem + lane_base + kColDP + c0 + j * 32, v);
         uint32_t w[16];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          const float4 dl = d4[ch * 8 + i];
-          const float a0 = p[ch * 32 + 4 * i + 0] * (__uint_as_float(v[4 * i + 0]) - dl.x);
-          const float a1 = p[ch * 32 + 4 * i + 1] * (__uint_as_float(v[4 * i + 1]) - dl.y);
-          const float a2 = p[ch * 32 + 4 * i + 2] * (__uint_as_float(v[4 * i + 2]) - dl.z);
-          const float a3 = p[ch * 32 + 4 * i + 3] * (__uint_as_float(v[4 * i + 3]) - dl.w);
+          const float4 dl = d4[j * 8 + i];
+          const float a0 = p[j * 32 + 4 * i + 0] * (__uint_as_float(v[4 * i + 0]) - dl.x);
+          const float a1 = p[j * 32 + 4 * i + 1] * (__uint_as_float(v[4 * i + 1]) - dl.y);
+          const float a2 = p[j * 32 + 4 * i + 2] * (__uint_as_float(v[4 * i + 2]) - dl.z);
+          const float a3 = p[j * 32 + 4 * i + 3] * (__uint_as_float(v[4 * i + 3]) - dl.w);
           w[2 * i] = pack_bf16x2(a0, a1);
           w[2 * i + 1] = pack_bf16x2(a2, a3);
           if constexpr (kPrecise) {
-            ds_lo[ch * 16 + 2 * i] = pack_bf16x2_residual(a0, a1, w[2 * i]);
-            ds_lo[ch * 16 + 2 * i + 1] = pack_bf16x2_residual(a2, a3, w[2 * i + 1]);
+            ds_lo[j * 16 + 2 * i] = pack_bf16x2_residual(a0, a1, w[2 * i]);
+            ds_lo[j * 16 + 2 * i + 1] = pack_bf16x2_residual(a2, a3, w[2 * i + 1]);
           }
         }
-        // Row r of the 128 x 128 bf16 tile: 64-column half (ch >> 1), 16-byte chunks
-        // (ch & 1) * 4 .. + 3, each stored at chunk index XOR (r & 7)  (128-byte swizzle).
-        const uint32_t row_addr = sDS + (ch >> 1) * 16384 + r * 128;
 #pragma unroll
         for (int c4 = 0; c4 < 4; ++c4) {
-          const uint32_t chunk = uint32_t((ch & 1) * 4 + c4) ^ uint32_t(r & 7);
+          const uint32_t chunk = uint32_t(j * 4 + c4) ^ uint32_t(r & 7);
           st_shared_v4(row_addr + chunk * 16, w[4 * c4], w[4 * c4 + 1], w[4 * c4 + 2], w[4 * c4 + 3]);
         }
       }
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(bar(B_DS_FULL));
+      if (leader) PSA_TRACE_MARK(it, 8);
       if constexpr (kPrecise) {
         // second term: same buffer, once the products of the first term have read it
         mbar_wait(bar(B_DS_EMPTY), dse_ph, wctx);
         dse_ph ^= 1;
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          const uint32_t row_addr = sDS + (ch >> 1) * 16384 + r * 128;
+        for (int j = 0; j < 2; ++j) {
 #pragma unroll
           for (int c4 = 0; c4 < 4; ++c4) {
-            const uint32_t chunk = uint32_t((ch & 1) * 4 + c4) ^ uint32_t(r & 7);
-            st_shared_v4(row_addr + chunk * 16, ds_lo[ch * 16 + 4 * c4], ds_lo[ch * 16 + 4 * c4 + 1],
-                         ds_lo[ch * 16 + 4 * c4 + 2], ds_lo[ch * 16 + 4 * c4 + 3]);
+            const uint32_t chunk = uint32_t(j * 4 + c4) ^ uint32_t(r & 7);
+            st_shared_v4(row_addr + chunk * 16, ds_lo[j * 16 + 4 * c4], ds_lo[j * 16 + 4 * c4 + 1],
+                         ds_lo[j * 16 + 4 * c4 + 2], ds_lo[j * 16 + 4 * c4 + 3]);
           }
         }
         fence_proxy_async_smem();
         mbar_arrive(bar(B_DS_FULL));
       }
 
-      s_lse[(st ^ 1) * kTile + ct] = nl2;
-      s_delta[(st ^ 1) * kTile + ct] = ndl;
-      named_bar_sync(1, 128);
+      store_stat(st ^ 1, next_stat);
+      named_bar_sync(1, 256);
     };
     for (int it = 0; it < n_it; ++it) {
       if (entry_of(it) & 2) iteration(it, std::true_type{});
       else iteration(it, std::false_type{});
     }
-
-    // ---- epilogue: dV, dK (scaled) -> bf16
-    mbar_wait(bar(B_DQ_FULL), (n_it - 1) & 1, wctx);
+    mbar_wait(bar(B_DONE), 0, wctx);
     tc_fence_after();
+
+    // ---- epilogue: this half's columns of dV and dK (scaled) -> bf16
     const int64_t row = int64_t(rec.row0) + r;
-    __nv_bfloat16* dv_row = prm.dv + (row * prm.Hkv + hk) * D;
-    __nv_bfloat16* dk_row = prm.dk + (row * prm.Hkv + hk) * D;
+    __nv_bfloat16* dv_row = prm.dv + (row * prm.Hkv + hk) * D + half * DH;
+    __nv_bfloat16* dk_row = prm.dk + (row * prm.Hkv + hk) * D + half * DH;
 #pragma unroll
     for (int which = 0; which < 2; ++which) {
       const float mul = which ? prm.scale : 1.f;
       __nv_bfloat16* dst_row = which ? dk_row : dv_row;
 #pragma unroll
-      for (int ch = 0; ch < D / 32; ++ch) {
+      for (int ch = 0; ch < DH / 32; ++ch) {
         uint32_t v[32];
-        tmem_ld32(tmem + lane_base + (which ? kColDK : kColDV) + ch * 32, v);
-        tc_wait_ld();
+        tmem_ld32_wait(tmem + lane_base + (which ? kColDK : kColDV) + half * DH + ch * 32, v);
         if (kv_valid) {
           uint4* dst = reinterpret_cast<uint4*>(dst_row + ch * 32);
 #pragma unroll
@@ -441,32 +503,69 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
     }
   } else {
-    // ------------------------------------------------------------ dQ drain, one query row per thread
+    // ------------------------------------------------------------ dQ drain: warps 12..15, one query row per thread
+    setmaxnreg_inc<152>();
     const int quarter = warp & 3;
     const int r = quarter * 32 + lane;
     const uint32_t lane_base = uint32_t(quarter * 32) << 16;
+    const bool leader = threadIdx.x == 384;
     const float sc = prm.scale;
+    const uint32_t stage0 = base + L::kDQS;
     for (int it = 0; it < n_it; ++it) {
       const int q0 = (entry_of(it) >> 2) * kTile;
-      const bool valid = q0 + r < rec.len;
-      float* dst_row = prm.dq_accum + ((int64_t(rec.ds) + q0 + r) * prm.Hq + head_of(it)) * D;
+      const int h = head_of(it);
       mbar_wait(bar(B_DQ_FULL), it & 1, wctx);
       tc_fence_after();
+      if (leader) PSA_TRACE_MARK(it, 9);
+      // Pull the whole row out of TMEM first and release the columns at once: the next dP^T
+      // is waiting for them.  Staging and reducing then proceed from registers, at the pace
+      // the reduce-adds are absorbed by L2.
+      uint32_t v[D];
 #pragma unroll
-      for (int ch = 0; ch < D / 32; ++ch) {
-        uint32_t v[32];
-        tmem_ld32(tmem + lane_base + kColDP + ch * 32, v);
-        tc_wait_ld();
-        if (valid) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i)
-            red_add_v4(dst_row + ch * 32 + 4 * i, __uint_as_float(v[4 * i]) * sc, __uint_as_float(v[4 * i + 1]) * sc,
-                       __uint_as_float(v[4 * i + 2]) * sc, __uint_as_float(v[4 * i + 3]) * sc);
-        }
-      }
+      for (int ch = 0; ch < D / 64; ++ch)
+        tmem_ld64_wait(tmem + lane_base + kColDP + ch * 64, reinterpret_cast<uint32_t(&)[64]>(v[ch * 64]));
+#ifndef PSA_EXPERIMENT_LATE_RELEASE
       tc_fence_before();
       mbar_arrive(bar(B_DQ_EMPTY));
+#endif
+#pragma unroll
+      for (int ch = 0; ch < D / 32; ++ch) {
+        const uint32_t stage = stage0 + (ch & 1) * L::kStageBytes;
+        // The reduce issued two chunks ago read this staging buffer: wait until it has.
+#ifdef PSA_EXPERIMENT_FULL_WAIT
+        if (leader) tma_wait_group<0>();
+#else
+        if (leader) tma_wait_group_read<1>();
+#endif
+        named_bar_sync(2, 128);
+        // Row r, 128 bytes, eight 16-byte chunks at index XOR (r & 7): the 128-byte swizzle the
+        // tensor map of dq_accum expects.  Rows past the sample's end hold exact zeros (their dS
+        // columns are masked), so adding them is harmless; rows past T are clipped by the TMA.
+        const uint32_t row_addr = stage + r * 128;
+#pragma unroll
+        for (int c4 = 0; c4 < 8; ++c4) {
+          const uint32_t chunk = uint32_t(c4) ^ uint32_t(r & 7);
+          st_shared_v4(row_addr + chunk * 16, __float_as_uint(__uint_as_float(v[ch * 32 + 4 * c4]) * sc),
+                       __float_as_uint(__uint_as_float(v[ch * 32 + 4 * c4 + 1]) * sc),
+                       __float_as_uint(__uint_as_float(v[ch * 32 + 4 * c4 + 2]) * sc),
+                       __float_as_uint(__uint_as_float(v[ch * 32 + 4 * c4 + 3]) * sc));
+        }
+        fence_proxy_async_smem();
+        named_bar_sync(2, 128);
+        if (leader) {
+#ifndef PSA_EXPERIMENT_SKIP_REDUCE
+          tma_reduce_add_3d(&tm_dq, stage, ch * 32, h, rec.ds + q0);
+#endif
+          tma_commit_group();
+        }
+      }
+#ifdef PSA_EXPERIMENT_LATE_RELEASE
+      tc_fence_before();
+      mbar_arrive(bar(B_DQ_EMPTY));
+#endif
+      if (leader) PSA_TRACE_MARK(it, 10);
     }
+    if (leader) tma_wait_group<0>();   // shared memory must outlive the last reduce
   }
 
   tc_fence_before();
@@ -529,9 +628,10 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
   float* dq_accum = reinterpret_cast<float*>(wsp + ws.dq_accum_off);
   float* delta = reinterpret_cast<float*>(wsp + ws.delta_off);
 
-  CUtensorMap tm_q, tm_k, tm_v, tm_do;
+  CUtensorMap tm_q, tm_k, tm_v, tm_do, tm_dq;
   if (!make_tile_map_bf16(&tm_q, q, T, plan->Hq, D) || !make_tile_map_bf16(&tm_k, k, T, plan->Hkv, D) ||
-      !make_tile_map_bf16(&tm_v, v, T, plan->Hkv, D) || !make_tile_map_bf16(&tm_do, d_o, T, plan->Hq, D))
+      !make_tile_map_bf16(&tm_v, v, T, plan->Hkv, D) || !make_tile_map_bf16(&tm_do, d_o, T, plan->Hq, D) ||
+      !make_tile_map(&tm_dq, dq_accum, T, plan->Hq, D, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, 32, 128))
     return PSA_ERR_CUDA;
   if (cudaFuncSetAttribute(psa_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kRequest) != cudaSuccess)
     return PSA_ERR_CUDA;
@@ -547,6 +647,7 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
   BwdParams prm;
   prm.tiles = plan->d_kv_tiles;
   prm.entries = plan->d_bwd_entries;
+  prm.cta_map = plan->d_bwd_cta_map;
   prm.lse = lse;
   prm.delta = delta;
   prm.dq_accum = dq_accum;
@@ -561,7 +662,7 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
   const unsigned grid = unsigned(plan->kv_tiles.size()) * unsigned(plan->Hkv);
   {
     ProfileScope prof(1, stream);
-    psa_bwd_kernel<D><<<grid, kBwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, tm_do, prm);
+    psa_bwd_kernel<D><<<grid, kBwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_dq, prm);
   }
   {
     const int64_t n_vec4 = n_rows * D / 4;
@@ -582,3 +683,10 @@ psa_status_t launch_bwd(const psa_plan_t* plan, const void* d_o, const void* q, 
 }
 
 }  // namespace psa
+
+#ifdef PSA_TRACE
+// Debug builds only: copies the 64 x 16 timestamp table of the last psa_bwd launch to the host.
+extern "C" int psa_trace_dump(long long* host_out) {
+  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_trace, sizeof(long long) * 64 * 16));
+}
+#endif

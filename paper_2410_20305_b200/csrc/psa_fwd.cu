@@ -175,8 +175,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {
         uint32_t v[32];
-        tmem_ld32(tmem + lane_base + kColS + ch * 32, v);
-        tc_wait_ld();
+        tmem_ld32_wait(tmem + lane_base + kColS + ch * 32, v);
 #pragma unroll
         for (int i = 0; i < 32; ++i) s[ch * 32 + i] = __uint_as_float(v[i]);
       }
@@ -211,8 +210,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
         for (int ch = 0; ch < D / 32; ++ch) {
           uint32_t v[32];
-          tmem_ld32(tmem + lane_base + kColO + ch * 32, v);
-          tc_wait_ld();
+          tmem_ld32_wait(tmem + lane_base + kColO + ch * 32, v);
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
           tmem_st32(tmem + lane_base + kColO + ch * 32, v);
@@ -257,8 +255,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
     for (int ch = 0; ch < D / 32; ++ch) {
       uint32_t v[32];
-      tmem_ld32(tmem + lane_base + kColO + ch * 32, v);
-      tc_wait_ld();
+      tmem_ld32_wait(tmem + lane_base + kColO + ch * 32, v);
       if (row_valid) {
         uint4* dst = reinterpret_cast<uint4*>(orow + ch * 32);
 #pragma unroll

@@ -32,6 +32,8 @@ struct psa_plan {
   size_t bwd_workspace_bytes = 0;
   std::vector<psa::TileRec> q_tiles, kv_tiles;   // sorted, longest list first
   std::vector<int32_t> fwd_entries, bwd_entries;
+  // Launch order of the backward CTAs: pairs (index into kv_tiles, kv head).
+  std::vector<int32_t> bwd_cta_map;
   // device copy (one allocation)
   int device = -1;
   void* d_blob = nullptr;
@@ -39,6 +41,7 @@ struct psa_plan {
   const psa::TileRec* d_kv_tiles = nullptr;
   const int32_t* d_fwd_entries = nullptr;
   const int32_t* d_bwd_entries = nullptr;
+  const int32_t* d_bwd_cta_map = nullptr;
 };
 
 namespace psa {

@@ -145,6 +145,33 @@ extern "C" psa_status_t psa_plan(const int32_t* cu_seqlens, const int32_t* prefi
   std::stable_sort(p->q_tiles.begin(), p->q_tiles.end(), longest_first);
   std::stable_sort(p->kv_tiles.begin(), p->kv_tiles.end(), longest_first);
   p->bwd_workspace_bytes = psa::bwd_workspace_layout(p->T, p->Hq, p->d).total;
+  // Backward CTA order.  Every CTA adds its dQ contributions into the fp32 accumulator rows of
+  // its sample and query-head group, so CTAs that share those rows are launched together: the
+  // rows then stay in L2 while they are being updated.  Samples with the most work first, then
+  // kv head, then the sample's key tiles, longest list first.
+  {
+    std::vector<int64_t> work(n_samples, 0);
+    std::vector<std::vector<int32_t>> tiles_of(n_samples);
+    std::vector<int32_t> sample_of_start(n_samples);
+    for (size_t t = 0; t < p->kv_tiles.size(); ++t) {
+      // the sample is found from its start row (cu_seqlens is increasing over non-empty samples)
+      const int32_t ds = p->kv_tiles[t].ds;
+      int s = int(std::upper_bound(cu_seqlens, cu_seqlens + n_samples + 1, ds) - cu_seqlens) - 1;
+      while (s + 1 < n_samples && cu_seqlens[s + 1] == ds) ++s;   // skip zero-length samples
+      work[s] += p->kv_tiles[t].list_cnt;
+      tiles_of[s].push_back(int32_t(t));                          // already longest first
+    }
+    std::vector<int> order(n_samples);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return work[a] > work[b]; });
+    p->bwd_cta_map.reserve(p->kv_tiles.size() * n_kv_heads * 2);
+    for (int s : order)
+      for (int hk = 0; hk < n_kv_heads; ++hk)
+        for (int32_t t : tiles_of[s]) {
+          p->bwd_cta_map.push_back(t);
+          p->bwd_cta_map.push_back(hk);
+        }
+  }
 
   if (!(flags & PSA_PLAN_HOST_ONLY)) {
     psa_status_t st = psa_plan_upload(p, stream);
@@ -165,7 +192,8 @@ extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
   const size_t b1 = up(p->kv_tiles.size() * sizeof(TileRec));
   const size_t b2 = up(p->fwd_entries.size() * sizeof(int32_t));
   const size_t b3 = up(p->bwd_entries.size() * sizeof(int32_t));
-  const size_t total = b0 + b1 + b2 + b3 + 256;
+  const size_t b4 = up(p->bwd_cta_map.size() * sizeof(int32_t));
+  const size_t total = b0 + b1 + b2 + b3 + b4 + 256;
   if (cudaGetDevice(&p->device) != cudaSuccess) return PSA_ERR_CUDA;
   void* blob = nullptr;
   if (cudaMalloc(&blob, total) != cudaSuccess) return PSA_ERR_CUDA;
@@ -176,6 +204,7 @@ extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
   std::memcpy(host.data() + b0, p->kv_tiles.data(), p->kv_tiles.size() * sizeof(TileRec));
   std::memcpy(host.data() + b0 + b1, p->fwd_entries.data(), p->fwd_entries.size() * sizeof(int32_t));
   std::memcpy(host.data() + b0 + b1 + b2, p->bwd_entries.data(), p->bwd_entries.size() * sizeof(int32_t));
+  std::memcpy(host.data() + b0 + b1 + b2 + b3, p->bwd_cta_map.data(), p->bwd_cta_map.size() * sizeof(int32_t));
   if (cudaMemcpyAsync(blob, host.data(), total, cudaMemcpyHostToDevice, cudaStream_t(stream)) != cudaSuccess ||
       cudaStreamSynchronize(cudaStream_t(stream)) != cudaSuccess) {
     cudaFree(blob);
@@ -187,6 +216,7 @@ extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
   p->d_kv_tiles = reinterpret_cast<const TileRec*>(b + b0);
   p->d_fwd_entries = reinterpret_cast<const int32_t*>(b + b0 + b1);
   p->d_bwd_entries = reinterpret_cast<const int32_t*>(b + b0 + b1 + b2);
+  p->d_bwd_cta_map = reinterpret_cast<const int32_t*>(b + b0 + b1 + b2 + b3);
   return PSA_OK;
 }
 
