@@ -57,7 +57,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -101,29 +101,35 @@ def whole_job_tflops(flops_per_replica, world, ms):
 
 
 def oracle_sample(pack, steps, warmup, target="bench"):
-    """Times the fp64 oracle, as it stands, on a bounded sample of the workload:
-    whole samples of the pack (attention is independent per sample) and one kv
-    group of 4 query heads.  Returns (useful TFLOP/s, description, cores, seconds per step)."""
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload: whole
+    samples of the pack (attention is independent per sample, which the oracle's own tests
+    pin) for one kv group of 4 query heads.  The baseline leg takes every sample of the
+    pack (1/8 of the workload's heads), the reference arm only the shortest sample because
+    it runs many steps.  Returns (useful TFLOP/s, description, cores, seconds per step)."""
     import torch
     from oracle import psa_oracle as orc
     from paper_2410_20305_b200 import workloads as wl
     order = np.argsort(pack.cu_seqlens[1:] - pack.cu_seqlens[:-1])
-    # the baseline leg takes the longest sample, the reference arm the shortest (it runs many steps)
-    s = int(order[-1] if target == "bench" else order[0])
-    P, C, R = int(pack.prefix_len[s]), int(pack.chosen_len[s]), int(pack.rejected_len[s])
-    sub = wl.pack_from_lengths("sample", [(P, C, R)], 4, 1, pack.head_dim)
-    q, k, v, d_o = (wl.to_f64(t) for t in wl.attention_inputs(sub, 2000, std=1.0))
-    mask = orc.packed_mask(sub.cu_seqlens, sub.prefix_len, sub.chosen_len, sub.rejected_len)
-    flops = 14.0 * pack.head_dim * 4 * orc.useful_pairs([P], [C], [R])
+    chosen = [int(x) for x in (order if target == "bench" else order[:1])]
+    subs, flops = [], 0.0
+    for s in chosen:
+        P, C, R = int(pack.prefix_len[s]), int(pack.chosen_len[s]), int(pack.rejected_len[s])
+        sub = wl.pack_from_lengths("sample", [(P, C, R)], 4, 1, pack.head_dim)
+        q, k, v, d_o = (wl.to_f64(t) for t in wl.attention_inputs(sub, 2000 + s, std=1.0))
+        mask = orc.packed_mask(sub.cu_seqlens, sub.prefix_len, sub.chosen_len, sub.rejected_len)
+        subs.append((q, k, v, d_o, mask))
+        flops += 14.0 * pack.head_dim * 4 * orc.useful_pairs([P], [C], [R])
     times = []
     for i in range(warmup + steps):
         t0 = time.perf_counter()
-        orc.attention_fwd(q, k, v, mask)
-        orc.attention_bwd(q, k, v, d_o, mask)
+        for q, k, v, d_o, mask in subs:
+            orc.attention_fwd(q, k, v, mask)
+            orc.attention_bwd(q, k, v, d_o, mask)
         if i >= warmup:
             times.append(time.perf_counter() - t0)
     sec = float(np.mean(times))
-    desc = "one sample of the pack (P=%d C=%d R=%d), 4 query heads / 1 kv head, fwd+bwd, dense fp64" % (P, C, R)
+    desc = "%d sample(s) of the pack (%d tokens), 4 query heads / 1 kv head, fwd+bwd, dense fp64 numpy" % (
+        len(chosen), int(sum(pack.cu_seqlens[s + 1] - pack.cu_seqlens[s] for s in chosen)))
     return flops / sec / 1e12, desc, torch.get_num_threads(), sec
 
 
@@ -151,6 +157,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-paired", action="store_true")
+    ap.add_argument("--no-logp", action="store_true", help="attention only (small footprint, for ncu captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -177,9 +184,10 @@ def main():
     T, Hq, Hkv, d = pack.total_tokens, pack.n_q_heads, pack.n_kv_heads, pack.head_dim
     q, k, v, d_o = (t.to(dev) for t in wl.attention_inputs(pack, 2000 + args.workload, std=1.0))
     gen = torch.Generator(device=dev).manual_seed(3000 + args.workload + rank)
-    logits = torch.empty((T, VOCAB), dtype=torch.bfloat16, device=dev)
-    for lo in range(0, T, 2048):   # N(0, variance 3), generated in slabs to bound the fp32 temporary
-        hi = min(T, lo + 2048)
+    n_logit_rows = 8 if args.no_logp else T
+    logits = torch.empty((n_logit_rows, VOCAB), dtype=torch.bfloat16, device=dev)
+    for lo in range(0, n_logit_rows, 2048):   # N(0, variance 3), generated in slabs to bound the fp32 temporary
+        hi = min(n_logit_rows, lo + 2048)
         logits[lo:hi] = (torch.randn((hi - lo, VOCAB), generator=gen, device=dev) * 3.0 ** 0.5).to(torch.bfloat16)
     tok = torch.randint(0, VOCAB, (T,), generator=gen, device=dev, dtype=torch.int32).cpu().numpy()
     targets, seg, fr, ft, fs = psa.logp_labels(tok, pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len)
@@ -209,7 +217,8 @@ def main():
         B.psa_fwd(plan, q, k, v, o=o, lse=lse, status=status)
         B.psa_bwd(plan, d_o, q, k, v, o, lse, dq=dq, dk=dk, dv=dv, workspace=ws, status=status)
         e_att1[i].record()
-        B.dpo_logp(logits, targets, seg_d, n_seg, fr, ft, fs, out=logp, status=status)
+        if not args.no_logp:
+            B.dpo_logp(logits, targets, seg_d, n_seg, fr, ft, fs, out=logp, status=status)
         e_lp1[i].record()
         return plan
 
@@ -230,7 +239,10 @@ def main():
         step(0, False)
         torch.cuda.synchronize()
         for name, pair in (("fwd", k_fwd), ("bwd", k_bwd), ("logp", k_lp)):
-            kernel_ms[name].append(pair[0].elapsed_time(pair[1]))
+            if name == "logp" and args.no_logp:
+                kernel_ms[name].append(float("nan"))
+            else:
+                kernel_ms[name].append(pair[0].elapsed_time(pair[1]))
     for which in range(3):
         B.psa_profile_events(which)
 
@@ -337,7 +349,7 @@ def main():
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": bwd_tflops / peaks["bf16_tflops"],
                      "peak_kind": "burst bf16 cuBLAS, of " + peaks["source"], "traffic": None},
         "clocks": clocks.summary(),
-        "gpu_launches": args.steps * 5,
+        "gpu_launches": args.steps * (4 if args.no_logp else 5),
         "paired_layout": paired,
         "paper_context": "paper reports 1.1-1.5x (1.3-1.6x with packing) end-to-end training speedups on 8xH100; context, not the target",
     }

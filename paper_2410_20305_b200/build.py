@@ -27,9 +27,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
-    if os.environ.get("PSA_EXPERIMENT"):   # timing experiments, results invalid
-        cmd += ["-D" + os.environ["PSA_EXPERIMENT"]]
-    if os.environ.get("PSA_TRACE"):   # debug build: hand-off timestamps of the backward kernel
+    if os.environ.get("PSA_TRACE"):   # debug build: SM-clock timestamps of the first CTA's hand-offs
+        # (read back with psa_trace_dump / psa_trace_dump_fwd, 64 iterations x 16 slots of int64)
         cmd += ["-DPSA_TRACE"]
     if verbose:
         cmd += ["-Xptxas", "-v"]

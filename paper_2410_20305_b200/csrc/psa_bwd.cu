@@ -524,19 +524,13 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
       for (int ch = 0; ch < D / 64; ++ch)
         tmem_ld64_wait(tmem + lane_base + kColDP + ch * 64, reinterpret_cast<uint32_t(&)[64]>(v[ch * 64]));
-#ifndef PSA_EXPERIMENT_LATE_RELEASE
       tc_fence_before();
       mbar_arrive(bar(B_DQ_EMPTY));
-#endif
 #pragma unroll
       for (int ch = 0; ch < D / 32; ++ch) {
         const uint32_t stage = stage0 + (ch & 1) * L::kStageBytes;
         // The reduce issued two chunks ago read this staging buffer: wait until it has.
-#ifdef PSA_EXPERIMENT_FULL_WAIT
-        if (leader) tma_wait_group<0>();
-#else
         if (leader) tma_wait_group_read<1>();
-#endif
         named_bar_sync(2, 128);
         // Row r, 128 bytes, eight 16-byte chunks at index XOR (r & 7): the 128-byte swizzle the
         // tensor map of dq_accum expects.  Rows past the sample's end hold exact zeros (their dS
@@ -553,16 +547,10 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         fence_proxy_async_smem();
         named_bar_sync(2, 128);
         if (leader) {
-#ifndef PSA_EXPERIMENT_SKIP_REDUCE
           tma_reduce_add_3d(&tm_dq, stage, ch * 32, h, rec.ds + q0);
-#endif
           tma_commit_group();
         }
       }
-#ifdef PSA_EXPERIMENT_LATE_RELEASE
-      tc_fence_before();
-      mbar_arrive(bar(B_DQ_EMPTY));
-#endif
       if (leader) PSA_TRACE_MARK(it, 10);
     }
     if (leader) tma_wait_group<0>();   // shared memory must outlive the last reduce

@@ -111,43 +111,11 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {  
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // All prior UMMAs of this thread arrive on the mbarrier when they have completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                        uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                        uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
-// 32 lanes x 32 consecutive 32-bit columns: thread = lane (row), v[c] = column c.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
 }
 // 32 consecutive columns of this thread's lane, loaded AND waited for inside one asm statement.
 // tcgen05.ld is asynchronous and its destination registers are not interlocked: if the load and
@@ -186,24 +154,17 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
 }
 
 // ---------------------------------------------------------------- descriptors
-// Shared-memory matrix descriptor, 128-byte swizzle, tile made of 8-row x 128-byte
-// atoms (1024 B, 1024-aligned).  Offsets are in bytes.
-//   K-major operand  (rows = M or N, 64 bf16 of K per row): sbo = bytes between 8-row groups; lbo unused.
-//   MN-major operand (rows = K, 64 bf16 of M/N per row):    sbo = bytes between 8-row (K) groups,
-//                                                           lbo = bytes between 64-element M/N chunks.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= uint64_t((smem_addr & 0x3FFFFu) >> 4);
-  d |= uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= uint64_t(1) << 46;  // descriptor version of this architecture
-  d |= uint64_t(2) << 61;  // 128-byte swizzle
-  return d;
-}
-// The same descriptor split into its 32-bit halves, so that the issuing thread (one thread,
-// every instruction on its critical path) advances an operand with one integer add:
-// the low word holds the start address and the LBO, the high word is a constant
-// (SBO = 1024 bytes, descriptor version, 128-byte swizzle).
+// Shared-memory matrix descriptor (64 bits), 128-byte swizzle, tile made of 8-row x 128-byte
+// atoms (1024 B, 1024-aligned):
+//   bits [0,14) start address >> 4, [16,30) leading byte offset >> 4, [32,46) stride byte
+//   offset >> 4, bit 46 descriptor version, bits [61,64) swizzle mode (2 = 128 bytes).
+//   K-major operand  (rows = M or N, 64 bf16 of K per row): SBO = bytes between 8-row groups; LBO unused.
+//   MN-major operand (rows = K, 64 bf16 of M/N per row):    SBO = bytes between 8-row (K) groups,
+//                                                           LBO = bytes between 64-element M/N chunks.
+// It is kept split into its 32-bit halves, so that the issuing thread (one thread, every
+// instruction on its critical path) advances an operand with one integer add: the low word
+// holds the start address and the LBO, the high word is a constant (SBO = 1024 bytes,
+// descriptor version, 128-byte swizzle).
 constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
 __device__ __forceinline__ uint32_t smem_desc_lo(uint32_t smem_addr, uint32_t lbo_bytes) {
   return ((smem_addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
@@ -247,15 +208,11 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, bool a_mn_m
 // Warpgroup register reallocation (all four warps of an aligned warpgroup must execute it).
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {
-#ifndef PSA_EXPERIMENT_NO_SETMAXNREG
   asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
-#endif
 }
 template <int N>
 __device__ __forceinline__ void setmaxnreg_dec() {
-#ifndef PSA_EXPERIMENT_NO_SETMAXNREG
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
-#endif
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {

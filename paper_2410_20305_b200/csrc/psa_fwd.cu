@@ -20,6 +20,16 @@
 #include "psa_tensormap.h"
 
 namespace psa {
+// Debug builds (-DPSA_TRACE) record SM-clock timestamps of the first CTA's hand-offs.
+#ifdef PSA_TRACE
+__device__ long long g_psa_trace_fwd[64 * 16];
+#define PSA_FWD_MARK(it, slot)                                                            \
+  do {                                                                                    \
+    if (blockIdx.x == 0 && (it) < 64) g_psa_trace_fwd[(it) * 16 + (slot)] = clock64();     \
+  } while (0)
+#else
+#define PSA_FWD_MARK(it, slot) do {} while (0)
+#endif
 namespace {
 
 using namespace dev;
@@ -47,7 +57,9 @@ struct FwdSmem {
   static constexpr int kBars = 3 * kTileBytes;        // 8 mbarriers
   static constexpr int kTmemSlot = kBars + 64;
   static constexpr int kAbort = kTmemSlot + 4;
-  static constexpr int kBytes = kBars + 128;
+  static constexpr int kEnt = kBars + 128;            // first kEntCap entries of the tile's list
+  static constexpr int kEntCap = 128;
+  static constexpr int kBytes = kEnt + kEntCap * 4;
   // Request enough that at most two CTAs fit on an SM: their TMEM allocations
   // (256 columns each) then always succeed without waiting.
   static constexpr int kRequest = (kBytes + 1024 > 100 * 1024) ? kBytes + 1024 : 100 * 1024;
@@ -75,8 +87,11 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const int h = blockIdx.x % prm.Hq;
   const int hk = h / (prm.Hq / prm.Hkv);
   const TileRec rec = prm.tiles[tile_idx];
-  const int32_t* ent = prm.entries + rec.list_off;
+  const int32_t* ent_g = prm.entries + rec.list_off;
   const int n_it = rec.list_cnt;
+  int32_t* s_ent = reinterpret_cast<int32_t*>(gen_base + L::kEnt);
+  // Every role reads the list entry of every iteration: keep the head of the list in shared memory.
+  auto ent = [&](int it) { return it < L::kEntCap ? s_ent[it] : ent_g[it]; };
   const WaitCtx wctx{abort_flag, prm.status};
 
   if (threadIdx.x == 0) {
@@ -91,6 +106,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     mbar_init(bar(BAR_O_FULL), 1);
     fence_mbar_init();
   }
+  if (int(threadIdx.x) < n_it && int(threadIdx.x) < L::kEntCap) s_ent[threadIdx.x] = ent_g[threadIdx.x];
   if (warp == 0) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
   }
@@ -108,7 +124,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_expect_tx(bar(BAR_Q_FULL), L::kTileBytes);
       for (int s = 0; s < L::kSub; ++s) tma_load_3d(sQ + s * L::kSubBytes, &tm_q, s * 64, h, rec.row0, bar(BAR_Q_FULL));
       for (int it = 0; it < n_it; ++it) {
-        const int krow = rec.ds + (ent[it] >> 2) * kTile;
+        const int krow = rec.ds + (ent(it) >> 2) * kTile;
         if (it > 0) mbar_wait(bar(BAR_K_EMPTY), (it - 1) & 1, wctx);
         mbar_expect_tx(bar(BAR_K_FULL), L::kTileBytes);
         for (int s = 0; s < L::kSub; ++s) tma_load_3d(sK + s * L::kSubBytes, &tm_k, s * 64, hk, krow, bar(BAR_K_FULL));
@@ -123,35 +139,42 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma_idesc_bf16(kTile, kTile, false, false);  // Q, K both K-major
       constexpr uint32_t idesc_o = umma_idesc_bf16(kTile, D, false, true);       // P (TMEM), V MN-major
+      // Low descriptor words (start address + LBO); the high word is a constant.
+      const uint32_t q_k = smem_desc_lo(sQ, 16), k_k = smem_desc_lo(sK, 16), v_mn = smem_desc_lo(sV, L::kSubBytes);
       mbar_wait(bar(BAR_Q_FULL), 0, wctx);
       for (int it = 0; it < n_it; ++it) {
+        PSA_FWD_MARK(it, 0);
         mbar_wait(bar(BAR_K_FULL), it & 1, wctx);
+        PSA_FWD_MARK(it, 1);
         // The S columns are also where P_{it-1} lives.  UMMAs issued by one thread execute in
         // issue order, so this S = Q K^T cannot overwrite P before the previous P V has read it.
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * L::kSubBytes + (kk & 3) * 32;
-          umma_ss(tmem + kColS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), idesc_s,
-                  kk > 0);
+          const uint32_t off = ((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4;
+          umma_ss_lo(tmem + kColS, q_k + off, k_k + off, idesc_s, kk > 0);
         }
         umma_commit(bar(BAR_K_EMPTY));
         umma_commit(bar(BAR_S_FULL));
+        PSA_FWD_MARK(it, 2);
         mbar_wait(bar(BAR_V_FULL), it & 1, wctx);
+        PSA_FWD_MARK(it, 3);
         mbar_wait(bar(BAR_P_FULL), it & 1, wctx);
+        PSA_FWD_MARK(it, 4);
         tc_fence_after();
         // PRECISE tiles carry P as two bf16 terms: columns [0,64) and [64,128) of the S region.
-        const int n_terms = (ent[it] & 2) ? 2 : 1;
+        const int n_terms = (ent(it) & 2) ? 2 : 1;
         for (int term = 0; term < n_terms; ++term) {
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk) {
             // A: 16 keys of P = 8 TMEM columns (two bf16 per column).  B: 16 key rows of V.
-            umma_ts(tmem + kColO, tmem + kColS + term * 64 + kk * 8,
-                    smem_desc_sw128(sV + kk * 2048, L::kSubBytes, 1024), idesc_o, (it > 0) || (kk > 0) || (term > 0));
+            umma_ts_lo(tmem + kColO, tmem + kColS + term * 64 + kk * 8, v_mn + kk * (2048 >> 4), idesc_o,
+                       (it > 0) || (kk > 0) || (term > 0));
           }
         }
         umma_commit(bar(BAR_V_EMPTY));
         umma_commit(bar(BAR_O_FULL));
+        PSA_FWD_MARK(it, 5);
       }
     }
     __syncwarp();
@@ -166,34 +189,80 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     float m_run = -INFINITY, l_run = 0.f;
 
     for (int it = 0; it < n_it; ++it) {
-      const int e = ent[it];
+      const int e = ent(it);
       const int k0 = (e >> 2) * kTile;
       const bool precise = (e & 2) != 0;
       mbar_wait(bar(BAR_S_FULL), it & 1, wctx);
       tc_fence_after();
-      float s[kTile];
-#pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
-        uint32_t v[32];
-        tmem_ld32_wait(tmem + lane_base + kColS + ch * 32, v);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) s[ch * 32 + i] = __uint_as_float(v[i]);
-      }
+      if (threadIdx.x == 64) PSA_FWD_MARK(it, 6);
+      // Allowed keys of this row in a PARTIAL tile, relative to the tile: [0, a) and [b, b + span).
+      int a = kTile, b = 0;
+      uint32_t span = 0;
       if (e & 1) {
-        // Allowed keys of this row, relative to the tile: [0, a) and [b, cc).
-        int a, b, cc;
-        if (q_local < rec.rs) { a = q_local + 1 - k0; b = 0; cc = 0; }
-        else { a = rec.cs - k0; b = rec.rs - k0; cc = q_local + 1 - k0; }
-        const uint32_t span = uint32_t(cc - b);
+        if (q_local < rec.rs) { a = q_local + 1 - k0; }
+        else { a = rec.cs - k0; b = rec.rs - k0; span = uint32_t(q_local + 1 - rec.rs); }
+      }
+      // Warp-uniform class of each 32-column chunk: 0 = every lane allows every column (no masking),
+      // 1 = mixed (mask per element), 2 = no lane allows any column (skipped: no load, no exponential).
+      // On a causal diagonal tile this skips 3/8 of the exponentials and masks only 1/4 of the columns.
+      uint32_t cls = 0;
+      if (e & 1) {
 #pragma unroll
-        for (int i = 0; i < kTile; ++i) {
-          const bool ok = (i < a) || (uint32_t(i - b) < span);
-          s[i] = ok ? s[i] : -INFINITY;
+        for (int ch = 0; ch < 4; ++ch) {
+          const int lo = ch * 32, hi = lo + 32;
+          const bool all_ok = (hi <= a) || (lo >= b && uint32_t(hi - b) <= span);
+          const bool none_ok = (lo >= a) && (span == 0u || hi <= b || (lo >= b && uint32_t(lo - b) >= span));
+          const uint32_t cc = __all_sync(0xffffffffu, all_ok) ? 0u : (__all_sync(0xffffffffu, none_ok) ? 2u : 1u);
+          cls |= cc << (2 * ch);
         }
       }
-      float mx = s[0];
+      auto chunk_class = [&](int ch) { return (cls >> (2 * ch)) & 3u; };
+      // The scores of the row are read from TMEM twice, 64 at a time (first for the row maximum,
+      // then for the exponentials), which keeps the live registers at half a row.
+      auto load_half = [&](int hf, float (&x)[64]) {
+        uint32_t v[64];
+        tmem_ld64_wait(tmem + lane_base + kColS + hf * 64, v);
+        if (!(e & 1)) {   // FULL tile: nothing to test
 #pragma unroll
-      for (int i = 1; i < kTile; ++i) mx = fmaxf(mx, s[i]);
+          for (int i = 0; i < 64; ++i) x[i] = __uint_as_float(v[i]);
+          return;
+        }
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub) {
+          const uint32_t cc = chunk_class(hf * 2 + sub);
+          if (cc == 1u) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int col = hf * 64 + sub * 32 + i;
+              const bool ok = (col < a) || (uint32_t(col - b) < span);
+              x[sub * 32 + i] = ok ? __uint_as_float(v[sub * 32 + i]) : -INFINITY;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) x[sub * 32 + i] = cc == 0u ? __uint_as_float(v[sub * 32 + i]) : -INFINITY;
+          }
+        }
+      };
+      auto half_skipped = [&](int hf) { return ((cls >> (4 * hf)) & 15u) == 10u; };   // both chunks of class 2
+      float mx;
+      {
+        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          if (half_skipped(hf)) continue;
+          float x[64];
+          load_half(hf, x);
+#pragma unroll
+          for (int i = 0; i < 64; i += 4) {
+            m4[0] = fmaxf(m4[0], x[i]);
+            m4[1] = fmaxf(m4[1], x[i + 1]);
+            m4[2] = fmaxf(m4[2], x[i + 2]);
+            m4[3] = fmaxf(m4[3], x[i + 3]);
+          }
+        }
+        mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+      }
+      if (threadIdx.x == 64) PSA_FWD_MARK(it, 7);
       const float m_new = fmaxf(m_run, mx);
       // Keep a stale maximum while it is within 2^8 of the true one: P stays <= 256
       // and the accumulator needs no rescaling.  (-inf) - (-inf) is NaN -> false.
@@ -216,32 +285,68 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           tmem_st32(tmem + lane_base + kColO + ch * 32, v);
         }
       }
+      if (threadIdx.x == 64) PSA_FWD_MARK(it, 8);
       const float mc = (m_run == -INFINITY) ? 0.f : m_run * c;
-      float sum = 0.f;
-      // P -> bf16 over the S columns ([0,64)); PRECISE tiles also store the rounding residual as a
-      // second bf16 term in columns [64,128).  Two instantiations keep the common path lean.
-      auto write_p = [&](auto precise_tag) {
-        constexpr bool kPrecise = decltype(precise_tag)::value;
+      float s4[4] = {0.f, 0.f, 0.f, 0.f};
+      if (!precise) {
+        // P -> bf16 over the S columns: the 64 values of half hf go to columns [32 hf, 32 hf + 32),
+        // which never reaches columns of S that are still to be read.
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          uint32_t v[32], vr[kPrecise ? 32 : 1];
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t v[32];
+          if (half_skipped(hf)) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = 0u;
+          } else {
+            float x[64];
+            load_half(hf, x);
+#pragma unroll
+            for (int sub = 0; sub < 2; ++sub) {
+              if (chunk_class(hf * 2 + sub) == 2u) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v[sub * 16 + i] = 0u;
+              } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                  const float p0 = ex2_approx(fmaf(x[sub * 32 + 2 * i], c, -mc));
+                  const float p1 = ex2_approx(fmaf(x[sub * 32 + 2 * i + 1], c, -mc));
+                  s4[i & 1] += p0;
+                  s4[2 + (i & 1)] += p1;
+                  v[sub * 16 + i] = pack_bf16x2(p0, p1);
+                }
+              }
+            }
+          }
+          tmem_st32(tmem + lane_base + kColS + hf * 32, v);
+        }
+      } else {
+        // PRECISE tiles also store the rounding residual as a second bf16 term in columns
+        // [64,128): all 128 scores are taken into registers before anything is written.
+        float x0[64], x1[64];
+        load_half(0, x0);
+        load_half(1, x1);
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t v[32], vr[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            const float p0 = ex2_approx(fmaf(s[ch * 64 + 2 * i], c, -mc));
-            const float p1 = ex2_approx(fmaf(s[ch * 64 + 2 * i + 1], c, -mc));
-            sum += p0 + p1;
+            const float p0 = ex2_approx(fmaf(hf ? x1[2 * i] : x0[2 * i], c, -mc));
+            const float p1 = ex2_approx(fmaf(hf ? x1[2 * i + 1] : x0[2 * i + 1], c, -mc));
+            s4[i & 1] += p0;
+            s4[2 + (i & 1)] += p1;
             v[i] = pack_bf16x2(p0, p1);
-            if constexpr (kPrecise) vr[i] = pack_bf16x2_residual(p0, p1, v[i]);
+            vr[i] = pack_bf16x2_residual(p0, p1, v[i]);
           }
-          tmem_st32(tmem + lane_base + kColS + ch * 32, v);
-          if constexpr (kPrecise) tmem_st32(tmem + lane_base + kColS + 64 + ch * 32, vr);
+          tmem_st32(tmem + lane_base + kColS + hf * 32, v);
+          tmem_st32(tmem + lane_base + kColS + 64 + hf * 32, vr);
         }
-      };
-      if (precise) write_p(std::true_type{}); else write_p(std::false_type{});
+      }
+      const float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
       l_run += sum;
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar(BAR_P_FULL));
+      if (threadIdx.x == 64) PSA_FWD_MARK(it, 9);
     }
 
     // ---- epilogue: O / l -> bf16, lse
@@ -320,3 +425,9 @@ psa_status_t launch_fwd(const psa_plan_t* plan, const void* q, const void* k, co
 }
 
 }  // namespace psa
+
+#ifdef PSA_TRACE
+extern "C" int psa_trace_dump_fwd(long long* host_out) {
+  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_trace_fwd, sizeof(long long) * 64 * 16));
+}
+#endif
