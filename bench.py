@@ -33,6 +33,9 @@ UNIT = "TFLOP/s"
 VOCAB = 128256            # logits width of the gather leg (bf16)
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes (read + write) of one psa_bwd_kernel launch, from the ncu capture summarised in
+# profiles/psa_bwd_kernel_llama3-8b.md (workload 1); other workloads have no capture.
+NCU_BWD_TRAFFIC_BYTES = {1: 997.3e6}
 
 
 def measured_peaks():
@@ -347,7 +350,9 @@ def main():
                     "dpo_logp_live_rows": live_rows, "dpo_logp_step_ms": lp_ms},
         "roofline": {"kernel": "psa_bwd_kernel<128>", "bound": "tensor", "achieved": bwd_tflops,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": bwd_tflops / peaks["bf16_tflops"],
-                     "peak_kind": "burst bf16 cuBLAS, of " + peaks["source"], "traffic": None},
+                     "peak_kind": "burst bf16 cuBLAS, of " + peaks["source"],
+                     "algorithmic_flops": flops_bwd, "algorithmic_bytes": 40960.0 * T if (Hq, Hkv, d) == (32, 8, 128) else None,
+                     "traffic": NCU_BWD_TRAFFIC_BYTES.get(args.workload)},
         "clocks": clocks.summary(),
         "gpu_launches": args.steps * (4 if args.no_logp else 5),
         "paired_layout": paired,

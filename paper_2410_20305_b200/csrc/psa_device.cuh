@@ -205,6 +205,14 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, bool a_mn_m
   return umma_idesc(M, N, kBF16, kBF16, a_mn_major, b_mn_major);
 }
 
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// Barrier among the n threads that name the same id (id 0 is the one __syncthreads uses).
+__device__ __forceinline__ void named_bar_sync(int id, int n) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+}
+
 // Warpgroup register reallocation (all four warps of an aligned warpgroup must execute it).
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {
