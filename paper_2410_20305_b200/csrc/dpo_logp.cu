@@ -1,5 +1,5 @@
 // dpo_logp: per-response summed log-probabilities (Section 2.1; responses are
-// recovered from their boundaries, Section 3.2).  HBM-bound: one CTA streams one
+// recovered from their boundaries, Section 3.2).  HBM-bound: one small CTA streams one
 // live logits row exactly once with 16-byte coalesced loads, keeps a running
 // (max, sum of exp) per thread in fp32, merges across the warp with shuffles and
 // across warps through shared memory, and adds  logit[target] - lse  into
@@ -16,7 +16,9 @@
 namespace psa {
 namespace {
 
-constexpr int kLogpThreads = 512;
+// 128 threads x 4 loads in flight measured best on B200 (6.86 TB/s on 8192 x 128256 bf16; 256 x 4: 6.71,
+// 512 x 4: 5.5, 1024 x 4: 4.6): small CTAs keep many rows in flight per SM and retire unevenly.
+constexpr int kLogpThreads = 128;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
