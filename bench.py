@@ -263,6 +263,27 @@ def main():
     if int(status.item()) != 0:
         raise SystemExit("device status word is %d: results invalid" % int(status.item()))
 
+    # ---- next step of the path (outside the timed step): DPO loss and its gradient into the logits
+    loss_bwd = None
+    if not args.no_logp and rank == 0:
+        dlogits = torch.empty_like(logits)
+        ref_lp = logp * 0.97
+        loss_t, coef = B.dpo_loss(logp, ref_lp, 0.1)
+        for _ in range(2):
+            B.dpo_logp_bwd(logits, targets, seg_d, coef, fr, ft, fs, dlogits=dlogits, status=status)
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(5):
+            B.dpo_logp_bwd(logits, targets, seg_d, coef, fr, ft, fs, dlogits=dlogits, status=status)
+        b.record()
+        torch.cuda.synchronize()
+        lb_ms = a.elapsed_time(b) / 5
+        lb_bytes = live_rows * VOCAB * 2 * 2 + (T - live_rows) * VOCAB * 2     # live rows read + written, dead rows zeroed
+        loss_bwd = {"dpo_loss": float(loss_t.item()), "dpo_logp_bwd_ms": lb_ms, "dpo_logp_bwd_gbs": lb_bytes / lb_ms / 1e6,
+                    "algorithmic_bytes": lb_bytes}
+        del dlogits
+
     # ---- the same kernels on the unshared paired layout (2n causal sequences)
     paired = None
     if not args.no_paired and rank == 0:
@@ -356,6 +377,7 @@ def main():
         "clocks": clocks.summary(),
         "gpu_launches": args.steps * (4 if args.no_logp else 5),
         "paired_layout": paired,
+        "next_rows": loss_bwd,
         "paper_context": "paper reports 1.1-1.5x (1.3-1.6x with packing) end-to-end training speedups on 8xH100; context, not the target",
     }
     if e2e:

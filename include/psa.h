@@ -223,6 +223,39 @@ psa_status_t dpo_logp(const void* logits, int32_t logits_dtype, int64_t n_rows, 
                       float* out, int32_t* device_status, void* stream);
 
 /*
+ * dpo_loss -- the DPO loss of Eq. 1 (Section 2.1) from the four summed log-probs per sample.
+ * The equation is printed as a ratio of logs; it is read as
+ *     loss = mean over samples s of  -log sigmoid(beta * margin_s),
+ *     margin_s = (policy[2s] - ref[2s]) - (policy[2s+1] - ref[2s+1])     (2s = chosen, 2s+1 = rejected).
+ *   policy_logps, ref_logps  device fp32 [2 * n_samples], as written by dpo_logp for the policy and
+ *                            the reference model
+ *   loss                     device fp32 [1] (out)
+ *   coef                     device fp32 [2 * n_samples] (out): d loss / d policy_logps
+ * Errors: INVALID_ARG, CUDA.
+ */
+psa_status_t dpo_loss(const float* policy_logps, const float* ref_logps, int32_t n_samples, float beta,
+                      float* loss, float* coef, void* stream);
+
+/*
+ * dpo_logp_bwd -- gradient of  sum_g coef[g] * out[g]  (out as written by dpo_logp) with respect
+ * to the logits:  dlogits[t][v] = sum over the labels (t, y, g) scored by row t of
+ *                 coef[g] * (1[v == y] - softmax(logits[t])[v]).
+ * Rows that score nothing are written as zeros and their logits are not read.
+ *   logits .. n_segments   exactly as for dpo_logp
+ *   coef                   device fp32 [n_segments], e.g. from dpo_loss
+ *   dlogits                device, same dtype, shape and row stride as logits (out); must not
+ *                          alias logits
+ *   device_status          as for dpo_logp; invalid labels are reported and skipped
+ * A row may carry at most 4 labels (its own and up to 3 forks); further ones are ignored.
+ * Errors: INVALID_ARG, ALIGNMENT, UNSUPPORTED, CUDA.
+ */
+psa_status_t dpo_logp_bwd(const void* logits, int32_t logits_dtype, int64_t n_rows, int64_t vocab,
+                          int64_t row_stride, const int32_t* targets, const int32_t* segment_ids,
+                          const int32_t* fork_rows, const int32_t* fork_targets,
+                          const int32_t* fork_segments, int32_t n_forks, int32_t n_segments,
+                          const float* coef, void* dlogits, int32_t* device_status, void* stream);
+
+/*
  * psa_profile_events -- measurement aid, no counterpart in the paper.  Registers a
  * pair of cudaEvent_t (passed as void*) that the next calls record on their stream
  * immediately before and after one chosen kernel, so that a benchmark can time that

@@ -26,6 +26,11 @@ Paper passages each function follows:
   from the packed row with the response boundaries (Section 3.2).
 * ``ideal_token_speedup`` / ``ideal_attention_speedup``: the two footnotes of
   Section 4.2 (2(p+c)/(p+2c) and 2(p+c)^2/(2(p+c)^2-p^2)).
+* ``dpo_loss`` / ``dpo_logp_grad``: Eq. 1 (Section 2.1).  The equation is printed as a
+  ratio of logs; it is read as the DPO loss of its cited source,
+  -log sigmoid(beta * [(lp_theta(chosen) - lp_ref(chosen)) - (lp_theta(rejected) - lp_ref(rejected))]),
+  averaged over the samples; its gradient with respect to the logits follows from
+  d log softmax(x)[y] / dx = onehot(y) - softmax(x).
 
 Parity pins (tests/test_oracle_*.py): the paired-format equivalence claimed in
 Section 3.1 checked against torch's own scaled_dot_product_attention and
@@ -285,3 +290,46 @@ def paired_response_logps(logits_fn, token_ids, cu_seqlens, prefix_len, chosen_l
                 if nxt >= P:
                     out[2 * s + which] += row_logprob(lg[i], tok[seq[nxt]])
     return out
+
+
+# --------------------------------------------------------------------------
+# DPO loss (Eq. 1) and its gradient back into the logits
+# --------------------------------------------------------------------------
+
+def dpo_loss(policy_logps, ref_logps, beta):
+    """Mean over the n samples of  -log sigmoid(beta * margin_s),
+    margin_s = (pol[2s] - ref[2s]) - (pol[2s+1] - ref[2s+1])   (entry 2s = chosen, 2s+1 = rejected).
+    Returns (loss, coef) with coef[g] = d loss / d policy_logps[g]."""
+    pol = np.asarray(policy_logps, dtype=np.float64)
+    ref = np.asarray(ref_logps, dtype=np.float64)
+    n = len(pol) // 2
+    margin = (pol[0::2] - ref[0::2]) - (pol[1::2] - ref[1::2])
+    z = float(beta) * margin
+    # -log sigmoid(z) = log(1 + exp(-z)), evaluated without overflow
+    loss_s = np.maximum(-z, 0.0) + np.log1p(np.exp(-np.abs(z)))
+    sig_neg = np.exp(-np.maximum(z, 0.0)) / (1.0 + np.exp(-np.abs(z)))      # sigmoid(-z)
+    coef = np.zeros(2 * n, dtype=np.float64)
+    coef[0::2] = -float(beta) * sig_neg / n
+    coef[1::2] = +float(beta) * sig_neg / n
+    return float(loss_s.mean()), coef
+
+
+def dpo_logp_grad(logits, targets, segment_ids, coef, fork_rows=(), fork_targets=(), fork_segments=()):
+    """d(sum_g coef[g] * out[g]) / d logits for out = dpo_logp(...): every scored (row t, label y,
+    response g) contributes coef[g] * (onehot(y) - softmax(logits[t])) to row t; rows that score
+    nothing get zeros."""
+    x = np.asarray(logits, dtype=np.float64)
+    d = np.zeros_like(x)
+    def add(t, y, g):
+        if g < 0:
+            return
+        m = x[t].max()
+        p = np.exp(x[t] - m)
+        p /= p.sum()
+        d[t] -= coef[g] * p
+        d[t, int(y)] += coef[g]
+    for t in range(x.shape[0]):
+        add(t, targets[t], int(segment_ids[t]))
+    for r, y, g in zip(fork_rows, fork_targets, fork_segments):
+        add(int(r), y, int(g))
+    return d

@@ -24,7 +24,7 @@ PSA_DEVSTAT_WAIT_EXPIRED, PSA_DEVSTAT_BAD_TARGET, PSA_DEVSTAT_BAD_SEGMENT = 1, 2
 EXPORTED_SYMBOLS = (
     "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
     "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp", "psa_profile_events",
-    "psa_bwd_static_scratch",
+    "psa_bwd_static_scratch", "dpo_loss", "dpo_logp_bwd",
 )
 
 
@@ -63,6 +63,8 @@ def load_library():
     lib.psa_bwd.argtypes = [vp] * 13
     lib.psa_bwd_static_scratch.argtypes = [vp] * 12
     lib.psa_profile_events.argtypes = [i32, vp, vp]
+    lib.dpo_loss.argtypes = [vp, vp, i32, f32, vp, vp, vp]
+    lib.dpo_logp_bwd.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     lib.dpo_logp.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     for name in EXPORTED_SYMBOLS:
         if name != "psa_status_string":
@@ -234,3 +236,39 @@ def psa_bwd_static_scratch(plan: Plan, d_o, q, k, v, o, lse, dq, dk, dv, status=
            load_library().psa_bwd_static_scratch(plan._h, _ptr(d_o), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
                                                  _ptr(dq), _ptr(dk), _ptr(dv), _ptr(status), _stream(stream)))
     return dq, dk, dv
+
+
+def dpo_loss(policy_logps, ref_logps, beta, stream=None):
+    """policy_logps, ref_logps fp32 CUDA [2n] (2s chosen, 2s+1 rejected) -> (loss fp32 [1], coef fp32 [2n])
+    with coef = d loss / d policy_logps; loss = mean_s -log sigmoid(beta * margin_s)."""
+    import torch
+    assert policy_logps.is_cuda and policy_logps.dtype == torch.float32 and policy_logps.is_contiguous()
+    assert ref_logps.shape == policy_logps.shape and ref_logps.dtype == torch.float32 and ref_logps.is_contiguous()
+    n = policy_logps.numel() // 2
+    loss = torch.empty(1, dtype=torch.float32, device=policy_logps.device)
+    coef = torch.empty(2 * n, dtype=torch.float32, device=policy_logps.device)
+    _check("dpo_loss", load_library().dpo_loss(_ptr(policy_logps), _ptr(ref_logps), n, float(beta), _ptr(loss),
+                                              _ptr(coef), _stream(stream)))
+    return loss, coef
+
+
+def dpo_logp_bwd(logits, targets, segment_ids, coef, fork_rows=None, fork_targets=None, fork_segments=None,
+                 dlogits=None, status=None, stream=None):
+    """Gradient of sum_g coef[g] * dpo_logp(...)[g] with respect to the logits; same dtype and
+    row stride as `logits`."""
+    import torch
+    assert logits.is_cuda and logits.dim() == 2 and logits.stride(1) == 1
+    dt = {torch.float32: PSA_DTYPE_F32, torch.bfloat16: PSA_DTYPE_BF16}[logits.dtype]
+    n_rows, vocab = logits.shape
+    n_forks = 0 if fork_rows is None else int(fork_rows.numel())
+    if not n_forks:
+        fork_rows = fork_targets = fork_segments = None
+    assert coef.is_cuda and coef.dtype == torch.float32 and coef.is_contiguous()
+    if dlogits is None:
+        dlogits = torch.empty_strided(logits.shape, logits.stride(), dtype=logits.dtype, device=logits.device)
+    assert dlogits.dtype == logits.dtype and dlogits.stride() == logits.stride()
+    _check("dpo_logp_bwd", load_library().dpo_logp_bwd(
+        _ptr(logits), dt, n_rows, vocab, logits.stride(0) if n_rows > 1 else vocab, _ptr(targets), _ptr(segment_ids),
+        _ptr(fork_rows), _ptr(fork_targets), _ptr(fork_segments), n_forks, int(coef.numel()), _ptr(coef),
+        _ptr(dlogits), _ptr(status), _stream(stream)))
+    return dlogits
