@@ -223,6 +223,24 @@ psa_status_t dpo_logp(const void* logits, int32_t logits_dtype, int64_t n_rows, 
                       float* out, int32_t* device_status, void* stream);
 
 /*
+ * psa_pack_ffd -- first-fit-decreasing packing of prefix-shared units into rows of a fixed
+ * packing length (Section 3.2: the packing unit is the shared prompt with both responses;
+ * Section 4.3.2: a first-fit-decreasing sampler, packing length = batch size x max unit length).
+ * Host only, no CUDA call.
+ *   unit_len      host int32 [n_units]: P + C + R of each sample (for the paired baseline layout
+ *                 pass 2P + C + R)
+ *   capacity      the packing length
+ *   bin_of_unit   host int32 [n_units] (out): index of the pack each unit goes to.  Units are
+ *                 taken from the longest to the shortest (ties: lower index first) and placed
+ *                 into the first pack, in order of creation, that still has room.
+ *   n_bins        host int32 (out): number of packs opened
+ * Errors: INVALID_ARG (null pointer, negative length, capacity <= 0), UNSUPPORTED (a unit is
+ * longer than the capacity; nothing is written).
+ */
+psa_status_t psa_pack_ffd(const int32_t* unit_len, int32_t n_units, int32_t capacity,
+                          int32_t* bin_of_unit, int32_t* n_bins);
+
+/*
  * dpo_loss -- the DPO loss of Eq. 1 (Section 2.1) from the four summed log-probs per sample.
  * The equation is printed as a ratio of logs; it is read as
  *     loss = mean over samples s of  -log sigmoid(beta * margin_s),

@@ -333,3 +333,53 @@ def dpo_logp_grad(logits, targets, segment_ids, coef, fork_rows=(), fork_targets
     for r, y, g in zip(fork_rows, fork_targets, fork_segments):
         add(int(r), y, int(g))
     return d
+
+
+# --------------------------------------------------------------------------
+# Packing of prefix-shared units (Section 3.2, Section 4.3.2: first-fit-decreasing)
+# --------------------------------------------------------------------------
+
+def ffd_pack(unit_lengths, capacity):
+    """First-fit-decreasing bin packing, the textbook algorithm: take the units from the
+    longest to the shortest (ties: lower index first) and put each into the first bin, in order
+    of creation, that still has room; open a new bin if none has.  Returns bin_of_unit
+    (list of bin indices).  A unit longer than the capacity is an error."""
+    order = sorted(range(len(unit_lengths)), key=lambda i: (-int(unit_lengths[i]), i))
+    free, bin_of = [], [None] * len(unit_lengths)
+    for i in order:
+        L = int(unit_lengths[i])
+        if L > capacity:
+            raise ValueError("unit %d of length %d exceeds the capacity %d" % (i, L, capacity))
+        for b in range(len(free)):
+            if free[b] >= L:
+                free[b] -= L
+                bin_of[i] = b
+                break
+        else:
+            free.append(capacity - L)
+            bin_of[i] = len(free) - 1
+    return bin_of
+
+
+def optimal_bin_count(unit_lengths, capacity):
+    """Fewest bins that hold all units, by exhaustive search (tiny inputs only)."""
+    items = sorted((int(x) for x in unit_lengths), reverse=True)
+    best = [len(items)]
+    def place(k, free):
+        if len(free) >= best[0]:
+            return
+        if k == len(items):
+            best[0] = len(free)
+            return
+        seen = set()
+        for b in range(len(free)):
+            if free[b] >= items[k] and free[b] not in seen:
+                seen.add(free[b])
+                free[b] -= items[k]
+                place(k + 1, free)
+                free[b] += items[k]
+        free.append(capacity - items[k])
+        place(k + 1, free)
+        free.pop()
+    place(0, [])
+    return best[0]

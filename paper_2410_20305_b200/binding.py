@@ -24,7 +24,7 @@ PSA_DEVSTAT_WAIT_EXPIRED, PSA_DEVSTAT_BAD_TARGET, PSA_DEVSTAT_BAD_SEGMENT = 1, 2
 EXPORTED_SYMBOLS = (
     "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
     "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp", "psa_profile_events",
-    "psa_bwd_static_scratch", "dpo_loss", "dpo_logp_bwd",
+    "psa_bwd_static_scratch", "dpo_loss", "dpo_logp_bwd", "psa_pack_ffd",
 )
 
 
@@ -64,6 +64,7 @@ def load_library():
     lib.psa_bwd_static_scratch.argtypes = [vp] * 12
     lib.psa_profile_events.argtypes = [i32, vp, vp]
     lib.dpo_loss.argtypes = [vp, vp, i32, f32, vp, vp, vp]
+    lib.psa_pack_ffd.argtypes = [vp, i32, i32, vp, C.POINTER(i32)]
     lib.dpo_logp_bwd.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     lib.dpo_logp.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     for name in EXPORTED_SYMBOLS:
@@ -272,3 +273,14 @@ def dpo_logp_bwd(logits, targets, segment_ids, coef, fork_rows=None, fork_target
         _ptr(fork_rows), _ptr(fork_targets), _ptr(fork_segments), n_forks, int(coef.numel()), _ptr(coef),
         _ptr(dlogits), _ptr(status), _stream(stream)))
     return dlogits
+
+
+def psa_pack_ffd(unit_len, capacity):
+    """First-fit-decreasing packing of units (P + C + R per sample) into packs of `capacity`
+    tokens.  Returns (bin_of_unit int32 [n], n_bins).  Host only."""
+    lens = _i32(unit_len)
+    bins = np.zeros(max(len(lens), 1), dtype=np.int32)
+    n_bins = C.c_int32()
+    _check("psa_pack_ffd", load_library().psa_pack_ffd(lens.ctypes.data, len(lens), int(capacity), bins.ctypes.data,
+                                                      C.byref(n_bins)))
+    return bins[:len(lens)], n_bins.value

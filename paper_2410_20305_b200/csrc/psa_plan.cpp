@@ -259,3 +259,43 @@ extern "C" psa_status_t psa_plan_export(const psa_plan_t* p, int32_t direction, 
   if (!e.empty()) std::memcpy(entries, e.data(), e.size() * sizeof(int32_t));
   return PSA_OK;
 }
+
+// First-fit-decreasing packing (Section 3.2 / 4.3.2).  The "first bin with room" query is
+// answered by a max segment tree over the bins' free space: O(n log n) for n units.
+extern "C" psa_status_t psa_pack_ffd(const int32_t* unit_len, int32_t n_units, int32_t capacity,
+                                     int32_t* bin_of_unit, int32_t* n_bins) {
+  if (n_units < 0 || capacity <= 0 || !n_bins || (n_units > 0 && (!unit_len || !bin_of_unit)))
+    return PSA_ERR_INVALID_ARG;
+  for (int i = 0; i < n_units; ++i) {
+    if (unit_len[i] < 0) return PSA_ERR_INVALID_ARG;
+    if (unit_len[i] > capacity) return PSA_ERR_UNSUPPORTED;
+  }
+  std::vector<int32_t> order(n_units);
+  std::iota(order.begin(), order.end(), 0);
+  std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return unit_len[a] > unit_len[b]; });
+  int leaves = 1;
+  while (leaves < std::max(n_units, 1)) leaves <<= 1;
+  std::vector<int32_t> tree(2 * leaves, 0);   // free space of bin b at tree[leaves + b]; unopened bins hold 0
+  int32_t opened = 0;
+  auto update = [&](int b, int32_t v) {
+    int node = leaves + b;
+    tree[node] = v;
+    for (node >>= 1; node >= 1; node >>= 1) tree[node] = std::max(tree[2 * node], tree[2 * node + 1]);
+  };
+  for (int32_t u : order) {
+    const int32_t len = unit_len[u];
+    int b;
+    if (opened > 0 && tree[1] >= len) {
+      int node = 1;
+      while (node < leaves) node = tree[2 * node] >= len ? 2 * node : 2 * node + 1;   // leftmost bin with room
+      b = node - leaves;
+    } else {
+      b = opened++;
+      update(b, capacity);
+    }
+    update(b, tree[leaves + b] - len);
+    bin_of_unit[u] = b;
+  }
+  *n_bins = opened;
+  return PSA_OK;
+}
