@@ -223,6 +223,32 @@ psa_status_t dpo_logp(const void* logits, int32_t logits_dtype, int64_t n_rows, 
                       float* out, int32_t* device_status, void* stream);
 
 /*
+ * psa_position_ids -- position ids of the shared layout (Section 3.1: the positions are set so
+ * that the sequences are the same as in the paired format): prompt and chosen tokens count on
+ * from 0 at the sample start, the j-th rejected token gets P + j.  Host only.
+ *   cu_seqlens, prefix_len, chosen_len, rejected_len, n_samples   as for psa_plan
+ *   position_ids   host int32 [T] (out)
+ * Errors: INVALID_ARG, INCONSISTENT_LENGTHS.
+ */
+psa_status_t psa_position_ids(const int32_t* cu_seqlens, const int32_t* prefix_len,
+                              const int32_t* chosen_len, const int32_t* rejected_len,
+                              int32_t n_samples, int32_t* position_ids);
+
+/*
+ * psa_rope -- rotary position embedding of a [n_tokens, n_heads, head_dim] bf16 tensor with
+ * per-token position ids, "rotate-half" convention (Llama family): with x = [x1 | x2] split at
+ * head_dim / 2 and angle_i = pos * rope_theta^(-2i / head_dim),
+ *     y1 = x1 cos - x2 sin,   y2 = x2 cos + x1 sin.
+ * q and k are rotated with it before psa_fwd (the kernels themselves are position-free).
+ *   x, y           device bf16; y may be x (in place)
+ *   position_ids   device int32 [n_tokens]
+ *   head_dim       multiple of 16, at most 256
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.
+ */
+psa_status_t psa_rope(const void* x, void* y, const int32_t* position_ids, int64_t n_tokens,
+                      int32_t n_heads, int32_t head_dim, float rope_theta, void* stream);
+
+/*
  * psa_pack_ffd -- first-fit-decreasing packing of prefix-shared units into rows of a fixed
  * packing length (Section 3.2: the packing unit is the shared prompt with both responses;
  * Section 4.3.2: a first-fit-decreasing sampler, packing length = batch size x max unit length).

@@ -383,3 +383,35 @@ def optimal_bin_count(unit_lengths, capacity):
         free.pop()
     place(0, [])
     return best[0]
+
+
+# --------------------------------------------------------------------------
+# Position ids of the shared layout (Section 3.1) and rotary embedding
+# --------------------------------------------------------------------------
+
+def position_ids(cu_seqlens, prefix_len, chosen_len, rejected_len):
+    """Section 3.1: positions are set so that each response sees the positions it would have
+    in the paired format: prompt and chosen tokens count on from the sample start, the
+    rejected tokens restart right after the prompt (position P + j for the j-th rejected token)."""
+    cu = np.asarray(cu_seqlens, dtype=np.int64)
+    pos = np.zeros(int(cu[-1]), dtype=np.int64)
+    for s in range(len(cu) - 1):
+        P, C, R = int(prefix_len[s]), int(chosen_len[s]), int(rejected_len[s])
+        ds = int(cu[s])
+        pos[ds:ds + P + C] = np.arange(P + C)
+        pos[ds + P + C:ds + P + C + R] = P + np.arange(R)
+    return pos
+
+
+def rope(x, pos, theta=10000.0):
+    """Rotary position embedding, "rotate-half" convention (the one Llama-family models use):
+    with x = [x1 | x2] split at d/2 and angle_i = pos * theta^(-2i/d),
+        y1 = x1 cos - x2 sin,   y2 = x2 cos + x1 sin.
+    x [T, H, d] float64, pos [T]."""
+    x = np.asarray(x, dtype=np.float64)
+    T, H, d = x.shape
+    inv_freq = float(theta) ** (-np.arange(0, d, 2, dtype=np.float64) / d)      # [d/2]
+    ang = np.asarray(pos, dtype=np.float64)[:, None] * inv_freq[None, :]        # [T, d/2]
+    cos, sin = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    x1, x2 = x[..., : d // 2], x[..., d // 2:]
+    return np.concatenate([x1 * cos - x2 * sin, x2 * cos + x1 * sin], axis=-1)

@@ -24,7 +24,7 @@ PSA_DEVSTAT_WAIT_EXPIRED, PSA_DEVSTAT_BAD_TARGET, PSA_DEVSTAT_BAD_SEGMENT = 1, 2
 EXPORTED_SYMBOLS = (
     "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
     "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp", "psa_profile_events",
-    "psa_bwd_static_scratch", "dpo_loss", "dpo_logp_bwd", "psa_pack_ffd",
+    "psa_bwd_static_scratch", "dpo_loss", "dpo_logp_bwd", "psa_pack_ffd", "psa_position_ids", "psa_rope",
 )
 
 
@@ -65,6 +65,8 @@ def load_library():
     lib.psa_profile_events.argtypes = [i32, vp, vp]
     lib.dpo_loss.argtypes = [vp, vp, i32, f32, vp, vp, vp]
     lib.psa_pack_ffd.argtypes = [vp, i32, i32, vp, C.POINTER(i32)]
+    lib.psa_position_ids.argtypes = [vp, vp, vp, vp, i32, vp]
+    lib.psa_rope.argtypes = [vp, vp, vp, i64, i32, i32, f32, vp]
     lib.dpo_logp_bwd.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     lib.dpo_logp.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     for name in EXPORTED_SYMBOLS:
@@ -284,3 +286,24 @@ def psa_pack_ffd(unit_len, capacity):
     _check("psa_pack_ffd", load_library().psa_pack_ffd(lens.ctypes.data, len(lens), int(capacity), bins.ctypes.data,
                                                       C.byref(n_bins)))
     return bins[:len(lens)], n_bins.value
+
+
+def psa_position_ids(cu_seqlens, prefix_len, chosen_len, rejected_len):
+    """Position ids int32 [T] of the shared layout: rejected tokens restart right after the prompt."""
+    cu, P, Cc, R = _i32(cu_seqlens), _i32(prefix_len), _i32(chosen_len), _i32(rejected_len)
+    out = np.zeros(max(int(cu[-1]), 1), dtype=np.int32)
+    _check("psa_position_ids", load_library().psa_position_ids(cu.ctypes.data, P.ctypes.data, Cc.ctypes.data,
+                                                              R.ctypes.data, len(P), out.ctypes.data))
+    return out[:int(cu[-1])]
+
+
+def psa_rope(x, position_ids, rope_theta=10000.0, out=None, stream=None):
+    """Rotary embedding (rotate-half convention) of x [T, H, d] bf16 CUDA with int32 CUDA position ids [T]."""
+    import torch
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.dim() == 3
+    assert position_ids.is_cuda and position_ids.dtype == torch.int32 and position_ids.numel() == x.shape[0]
+    if out is None:
+        out = torch.empty_like(x)
+    _check("psa_rope", load_library().psa_rope(_ptr(x), _ptr(out), _ptr(position_ids), x.shape[0], x.shape[1],
+                                              x.shape[2], float(rope_theta), _stream(stream)))
+    return out

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpsa.so")
-SOURCES = ["psa_plan.cpp", "psa_api.cu", "psa_fwd.cu", "psa_bwd.cu", "psa_bwd_static.cu", "dpo_logp.cu", "dpo_loss.cu"]
+SOURCES = ["psa_plan.cpp", "psa_api.cu", "psa_fwd.cu", "psa_bwd.cu", "psa_bwd_static.cu", "dpo_logp.cu", "dpo_loss.cu", "psa_rope.cu"]
 
 
 def _stale() -> bool:
