@@ -2,9 +2,10 @@
 // read as  -log sigmoid(beta * [(lp_theta(c) - lp_ref(c)) - (lp_theta(r) - lp_ref(r))]),
 // averaged over the samples) and its gradient back into the logits,
 //     dlogits[t][v] = sum over labels (t, y, g) scored by row t of  coef[g] * (1[v == y] - softmax(logits[t])[v]).
-// dpo_logp_bwd is HBM-bound: every live row is read once from DRAM (the second sweep hits L2:
-// at most two 512-thread CTAs per SM keep the rows in flight below the L2 capacity) and written
-// once; rows that score nothing are only written (zeros).
+// dpo_logp_bwd is HBM-bound: every live row is read once from DRAM (the second sweep is meant to
+// hit L2: one 1024-thread CTA per SM keeps 148 rows in flight, the first sweep loads with an
+// evict-last policy, the second with evict-first, and the gradient is written with streaming
+// stores) and written once; rows that score nothing are only written (zeros).
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -17,7 +18,7 @@
 namespace psa {
 namespace {
 
-constexpr int kBwdLogpThreads = 512;
+constexpr int kBwdLogpThreads = 1024;   // one CTA per SM: 148 rows (38 MB) in flight, well inside L2
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -26,9 +27,18 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ uint4 ld_16(const uint4* p) {
+__device__ __forceinline__ uint4 ld_16_keep(const uint4* p) {   // first sweep: ask L2 to keep the line for the second
   uint4 v;
-  asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  asm volatile("ld.global.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
+  return v;
+}
+__device__ __forceinline__ uint4 ld_16_last(const uint4* p) {   // second sweep: the line is not needed again
+  uint4 v;
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
   return v;
 }
 __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
@@ -107,7 +117,7 @@ __global__ void dpo_loss_kernel(const float* __restrict__ pol, const float* __re
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kBwdLogpThreads, 2)
+__global__ void __launch_bounds__(kBwdLogpThreads, 1)
 dpo_logp_bwd_kernel(const T* __restrict__ logits, int64_t vocab, int64_t row_stride, const int32_t* __restrict__ targets,
                     const int32_t* __restrict__ segment_ids, const int32_t* __restrict__ fork_rows,
                     const int32_t* __restrict__ fork_targets, const int32_t* __restrict__ fork_segments,
@@ -152,7 +162,7 @@ dpo_logp_bwd_kernel(const T* __restrict__ logits, int64_t vocab, int64_t row_str
   MaxSum acc{-INFINITY, 0.f};
   for (int64_t i = threadIdx.x; i < n_vec; i += kBwdLogpThreads) {
     float y[E];
-    Elem<T>::unpack(ld_16(xv + i), y);
+    Elem<T>::unpack(ld_16_keep(xv + i), y);
     float mx = y[0];
 #pragma unroll
     for (int j = 1; j < E; ++j) mx = fmaxf(mx, y[j]);
@@ -194,7 +204,7 @@ dpo_logp_bwd_kernel(const T* __restrict__ logits, int64_t vocab, int64_t row_str
   // ---- sweep 2: -csum * softmax, streamed out (the row comes from L2 this time)
   for (int64_t i = threadIdx.x; i < n_vec; i += kBwdLogpThreads) {
     float y[E];
-    Elem<T>::unpack(ld_16(xv + i), y);
+    Elem<T>::unpack(ld_16_last(xv + i), y);
 #pragma unroll
     for (int j = 0; j < E; ++j) y[j] = -csum * ex2_approx(fmaf(y[j], kLog2e, -lse2));
     st_stream(reinterpret_cast<uint4*>(dx) + i, Elem<T>::pack(y));

@@ -1,14 +1,18 @@
 // psa_fwd: attention forward under the prefix-sharing mask with packing
 // (Algorithm 3; Section 3.1), one CTA per (query tile, query head).
 //
-// Warp roles (192 threads):
-//   warp 0      TMA producer: Q once, then K_j and V_j of every live key tile
-//   warp 1      UMMA issuer:  S = Q K_j^T  and  O += P V_j  (tcgen05, accumulators in TMEM)
-//   warps 2..5  softmax: one thread per query row; S is read from TMEM, masked in
-//               registers when the tile is PARTIAL, turned into P = exp2(S*c - m*c)
-//               in fp32 and written back to TMEM as bf16 (over S) for the second UMMA.
-// Two CTAs share an SM (96 KB of shared memory and 256 TMEM columns each for
-// head_dim 128), so one CTA's softmax overlaps the other's UMMAs.
+// Warp roles (384 threads = 3 warpgroups):
+//   warp 0       TMA producer: Q once, then K_j and V_j of every live key tile
+//   warp 1       UMMA issuer:  S = Q K_j^T  and  O += P V_j  (tcgen05, accumulators in TMEM)
+//   warps 2, 3   idle (they complete the first warpgroup, which gives its registers away)
+//   warps 4..11  softmax: two threads per query row, one for each half of the 128 key columns.
+//                S is read from TMEM, masked in registers when the tile is PARTIAL, turned into
+//                P = exp2(S*c - m*c) in fp32 and written back to TMEM as bf16 (over the thread's
+//                own S columns) for the second UMMA.  The two halves of a row exchange their
+//                maxima through shared memory.
+// Two CTAs share an SM (100 KB of shared memory and 256 TMEM columns each for head_dim 128), so
+// one CTA's softmax overlaps the other's UMMAs, and with eight softmax warps per CTA every SM
+// sub-partition has two warps feeding its exponential unit even when only one CTA is in that phase.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -34,7 +38,11 @@ namespace {
 
 using namespace dev;
 
-constexpr int kFwdThreads = 192;
+constexpr int kFwdThreads = 384;
+constexpr int kSoftmaxThreads = 256;
+// Register split of the 80 per thread the launch bound allows: the first warpgroup (producer,
+// issuer) gives registers to the two softmax warpgroups.
+constexpr int kRegsWg0 = 40, kRegsSoftmax = 96;
 constexpr uint32_t kTmemCols = 256;   // S: columns [0,128), O: columns [128, 128+D)
 constexpr uint32_t kColS = 0, kColO = 128;
 
@@ -59,7 +67,8 @@ struct FwdSmem {
   static constexpr int kAbort = kTmemSlot + 4;
   static constexpr int kEnt = kBars + 128;            // first kEntCap entries of the tile's list
   static constexpr int kEntCap = 128;
-  static constexpr int kBytes = kEnt + kEntCap * 4;
+  static constexpr int kXchg = kEnt + kEntCap * 4;    // float [2 parities][2 halves][128 rows]
+  static constexpr int kBytes = kXchg + 2 * 2 * kTile * 4;
   // Request enough that at most two CTAs fit on an SM: their TMEM allocations
   // (256 columns each) then always succeed without waiting.
   static constexpr int kRequest = (kBytes + 1024 > 100 * 1024) ? kBytes + 1024 : 100 * 1024;
@@ -102,7 +111,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     mbar_init(bar(BAR_K_EMPTY), 1);
     mbar_init(bar(BAR_V_EMPTY), 1);
     mbar_init(bar(BAR_S_FULL), 1);
-    mbar_init(bar(BAR_P_FULL), 128);
+    mbar_init(bar(BAR_P_FULL), kSoftmaxThreads);
     mbar_init(bar(BAR_O_FULL), 1);
     fence_mbar_init();
   }
@@ -115,7 +124,9 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
 
-  if (warp == 0) {
+  if (warp < 4) {
+   setmaxnreg_dec<kRegsWg0>();
+   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
       tma_prefetch_desc(&tm_q);
@@ -134,7 +145,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
+   } else if (warp == 1) {
     // ------------------------------------------------------------ UMMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma_idesc_bf16(kTile, kTile, false, false);  // Q, K both K-major
@@ -162,13 +173,14 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         mbar_wait(bar(BAR_P_FULL), it & 1, wctx);
         PSA_FWD_MARK(it, 4);
         tc_fence_after();
-        // PRECISE tiles carry P as two bf16 terms: columns [0,64) and [64,128) of the S region.
+        // P of key half hf lies in columns [64 hf, 64 hf + 32) of the S region (two bf16 per column);
+        // PRECISE tiles carry a second bf16 term in columns [64 hf + 32, 64 hf + 64).
         const int n_terms = (ent(it) & 2) ? 2 : 1;
         for (int term = 0; term < n_terms; ++term) {
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk) {
             // A: 16 keys of P = 8 TMEM columns (two bf16 per column).  B: 16 key rows of V.
-            umma_ts_lo(tmem + kColO, tmem + kColS + term * 64 + kk * 8, v_mn + kk * (2048 >> 4), idesc_o,
+            umma_ts_lo(tmem + kColO, tmem + kColS + (kk >> 2) * 64 + term * 32 + (kk & 3) * 8, v_mn + kk * (2048 >> 4), idesc_o,
                        (it > 0) || (kk > 0) || (term > 0));
           }
         }
@@ -178,15 +190,30 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
     }
     __syncwarp();
+   }
   } else {
-    // ------------------------------------------------------------ softmax, one row per thread
+    // ------------------------------------------------------------ softmax, two threads per row
+    setmaxnreg_inc<kRegsSoftmax>();
     const int quarter = warp & 3;                 // TMEM lanes this warp may touch
+    const int hfz = (warp - 4) >> 2;              // which half of the key columns this thread owns
     const int r = quarter * 32 + lane;            // row within the tile
     const uint32_t lane_base = uint32_t(quarter * 32) << 16;
+    const uint32_t col_s = kColS + 64u * hfz;     // this thread's 64 S columns; its P goes over them
     const int q_local = rec.local0 + r;
     const bool row_valid = q_local < rec.len;
     const float c = prm.scale_log2;
-    float m_run = -INFINITY, l_run = 0.f;
+    float* xchg = reinterpret_cast<float*>(gen_base + L::kXchg);
+    float m_run = -INFINITY, l_run = 0.f;         // l_run: this thread's half of the row sum
+    // Barrier of the two warps that share a row quarter (ids 1..4, immediate so that the kernel
+    // is known to use five barriers, not all sixteen).
+    auto pair_sync = [&]() {
+      switch (quarter) {
+        case 0: asm volatile("bar.sync 1, 64;" ::: "memory"); break;
+        case 1: asm volatile("bar.sync 2, 64;" ::: "memory"); break;
+        case 2: asm volatile("bar.sync 3, 64;" ::: "memory"); break;
+        default: asm volatile("bar.sync 4, 64;" ::: "memory"); break;
+      }
+    };
 
     for (int it = 0; it < n_it; ++it) {
       const int e = ent(it);
@@ -194,7 +221,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const bool precise = (e & 2) != 0;
       mbar_wait(bar(BAR_S_FULL), it & 1, wctx);
       tc_fence_after();
-      if (threadIdx.x == 64) PSA_FWD_MARK(it, 6);
+      if (threadIdx.x == 128) PSA_FWD_MARK(it, 6);
       // Allowed keys of this row in a PARTIAL tile, relative to the tile: [0, a) and [b, b + span).
       int a = kTile, b = 0;
       uint32_t span = 0;
@@ -202,58 +229,48 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (q_local < rec.rs) { a = q_local + 1 - k0; }
         else { a = rec.cs - k0; b = rec.rs - k0; span = uint32_t(q_local + 1 - rec.rs); }
       }
-      // Warp-uniform class of each 32-column chunk: 0 = every lane allows every column (no masking),
-      // 1 = mixed (mask per element), 2 = no lane allows any column (skipped: no load, no exponential).
-      // On a causal diagonal tile this skips 3/8 of the exponentials and masks only 1/4 of the columns.
+      // Warp-uniform class of this warp's two 32-column chunks: 0 = every lane allows every column
+      // (no masking), 1 = mixed (mask per element), 2 = no lane allows any column (skipped: no load,
+      // no exponential).  On a causal diagonal tile this skips 3/8 of the exponentials.
       uint32_t cls = 0;
       if (e & 1) {
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          const int lo = ch * 32, hi = lo + 32;
+        for (int sub = 0; sub < 2; ++sub) {
+          const int lo = hfz * 64 + sub * 32, hi = lo + 32;
           const bool all_ok = (hi <= a) || (lo >= b && uint32_t(hi - b) <= span);
           const bool none_ok = (lo >= a) && (span == 0u || hi <= b || (lo >= b && uint32_t(lo - b) >= span));
           const uint32_t cc = __all_sync(0xffffffffu, all_ok) ? 0u : (__all_sync(0xffffffffu, none_ok) ? 2u : 1u);
-          cls |= cc << (2 * ch);
+          cls |= cc << (2 * sub);
         }
       }
-      auto chunk_class = [&](int ch) { return (cls >> (2 * ch)) & 3u; };
-      // The scores of the row are read from TMEM twice, 64 at a time (first for the row maximum,
-      // then for the exponentials), which keeps the live registers at half a row.
-      auto load_half = [&](int hf, float (&x)[64]) {
-        uint32_t v[64];
-        tmem_ld64_wait(tmem + lane_base + kColS + hf * 64, v);
-        if (!(e & 1)) {   // FULL tile: nothing to test
+      auto chunk_class = [&](int sub) { return (cls >> (2 * sub)) & 3u; };
+      // The thread's scores are read from TMEM twice, 32 at a time (first for the row maximum,
+      // then for the exponentials), which keeps the live registers small.
+      auto load_chunk = [&](int sub, float (&x)[32]) {
+        uint32_t v[32];
+        tmem_ld32_wait(tmem + lane_base + col_s + sub * 32, v);
+        if (chunk_class(sub) == 1u) {
 #pragma unroll
-          for (int i = 0; i < 64; ++i) x[i] = __uint_as_float(v[i]);
-          return;
-        }
-#pragma unroll
-        for (int sub = 0; sub < 2; ++sub) {
-          const uint32_t cc = chunk_class(hf * 2 + sub);
-          if (cc == 1u) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const int col = hf * 64 + sub * 32 + i;
-              const bool ok = (col < a) || (uint32_t(col - b) < span);
-              x[sub * 32 + i] = ok ? __uint_as_float(v[sub * 32 + i]) : -INFINITY;
-            }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) x[sub * 32 + i] = cc == 0u ? __uint_as_float(v[sub * 32 + i]) : -INFINITY;
+          for (int i = 0; i < 32; ++i) {
+            const int col = hfz * 64 + sub * 32 + i;
+            const bool ok = (col < a) || (uint32_t(col - b) < span);
+            x[i] = ok ? __uint_as_float(v[i]) : -INFINITY;
           }
+        } else {   // class 0; callers never use the values of a class-2 chunk
+#pragma unroll
+          for (int i = 0; i < 32; ++i) x[i] = __uint_as_float(v[i]);
         }
       };
-      auto half_skipped = [&](int hf) { return ((cls >> (4 * hf)) & 15u) == 10u; };   // both chunks of class 2
       float mx;
       {
         float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          if (half_skipped(hf)) continue;
-          float x[64];
-          load_half(hf, x);
+        for (int sub = 0; sub < 2; ++sub) {
+          if (chunk_class(sub) == 2u) continue;
+          float x[32];
+          load_chunk(sub, x);
 #pragma unroll
-          for (int i = 0; i < 64; i += 4) {
+          for (int i = 0; i < 32; i += 4) {
             m4[0] = fmaxf(m4[0], x[i]);
             m4[1] = fmaxf(m4[1], x[i + 1]);
             m4[2] = fmaxf(m4[2], x[i + 2]);
@@ -262,10 +279,20 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
       }
-      if (threadIdx.x == 64) PSA_FWD_MARK(it, 7);
+      // Row maximum over both halves: the two threads of a row trade maxima through shared memory
+      // (slots alternate with the iteration parity, so a slot is rewritten only after the partner
+      // has passed the next barrier, hence read it).
+      {
+        float* slot = xchg + (it & 1) * 2 * kTile;
+        slot[hfz * kTile + r] = mx;
+        pair_sync();
+        mx = fmaxf(mx, slot[(hfz ^ 1) * kTile + r]);
+      }
+      if (threadIdx.x == 128) PSA_FWD_MARK(it, 7);
       const float m_new = fmaxf(m_run, mx);
       // Keep a stale maximum while it is within 2^8 of the true one: P stays <= 256
       // and the accumulator needs no rescaling.  (-inf) - (-inf) is NaN -> false.
+      // Both threads of a row see the same maxima, hence take the same decision.
       const bool grow = (m_new - m_run) * c > 8.0f;
       float alpha = 1.f;
       if (grow) {
@@ -276,69 +303,72 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (it > 0 && __any_sync(0xffffffffu, grow)) {
         mbar_wait(bar(BAR_O_FULL), (it - 1) & 1, wctx);
         tc_fence_after();
+        // Each thread rescales its half of the accumulator's columns.
 #pragma unroll
-        for (int ch = 0; ch < D / 32; ++ch) {
+        for (int ch = 0; ch < D / 64; ++ch) {
           uint32_t v[32];
-          tmem_ld32_wait(tmem + lane_base + kColO + ch * 32, v);
+          const uint32_t col = kColO + hfz * (D / 2) + ch * 32;
+          tmem_ld32_wait(tmem + lane_base + col, v);
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-          tmem_st32(tmem + lane_base + kColO + ch * 32, v);
+          tmem_st32(tmem + lane_base + col, v);
         }
       }
-      if (threadIdx.x == 64) PSA_FWD_MARK(it, 8);
+      if (threadIdx.x == 128) PSA_FWD_MARK(it, 8);
       const float mc = (m_run == -INFINITY) ? 0.f : m_run * c;
       float s4[4] = {0.f, 0.f, 0.f, 0.f};
       if (!precise) {
-        // P -> bf16 over the S columns: the 64 values of half hf go to columns [32 hf, 32 hf + 32),
-        // which never reaches columns of S that are still to be read.
+        // P -> bf16 over the thread's own S columns: the 32 values of chunk sub go to columns
+        // [16 sub, 16 sub + 16) of them, which never reaches a column that is still to be read.
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          uint32_t v[32];
-          if (half_skipped(hf)) {
+        for (int sub = 0; sub < 2; ++sub) {
+          uint32_t v[16];
+          if (chunk_class(sub) == 2u) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = 0u;
+            for (int i = 0; i < 16; ++i) v[i] = 0u;
           } else {
-            float x[64];
-            load_half(hf, x);
+            float x[32];
+            load_chunk(sub, x);
 #pragma unroll
-            for (int sub = 0; sub < 2; ++sub) {
-              if (chunk_class(hf * 2 + sub) == 2u) {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) v[sub * 16 + i] = 0u;
-              } else {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                  const float p0 = ex2_approx(fmaf(x[sub * 32 + 2 * i], c, -mc));
-                  const float p1 = ex2_approx(fmaf(x[sub * 32 + 2 * i + 1], c, -mc));
-                  s4[i & 1] += p0;
-                  s4[2 + (i & 1)] += p1;
-                  v[sub * 16 + i] = pack_bf16x2(p0, p1);
-                }
-              }
+            for (int i = 0; i < 16; ++i) {
+              const float p0 = ex2_approx(fmaf(x[2 * i], c, -mc));
+              const float p1 = ex2_approx(fmaf(x[2 * i + 1], c, -mc));
+              s4[i & 1] += p0;
+              s4[2 + (i & 1)] += p1;
+              v[i] = pack_bf16x2(p0, p1);
             }
           }
-          tmem_st32(tmem + lane_base + kColS + hf * 32, v);
+          tmem_st16(tmem + lane_base + col_s + sub * 16, v);
         }
       } else {
         // PRECISE tiles also store the rounding residual as a second bf16 term in columns
-        // [64,128): all 128 scores are taken into registers before anything is written.
-        float x0[64], x1[64];
-        load_half(0, x0);
-        load_half(1, x1);
+        // [32,64) of the thread's own: all 64 scores are taken into registers before anything
+        // is written.
+        float x0[32], x1[32];
+        load_chunk(0, x0);
+        load_chunk(1, x1);
+        if (chunk_class(0) == 2u) {
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          uint32_t v[32], vr[32];
+          for (int i = 0; i < 32; ++i) x0[i] = -INFINITY;
+        }
+        if (chunk_class(1) == 2u) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float p0 = ex2_approx(fmaf(hf ? x1[2 * i] : x0[2 * i], c, -mc));
-            const float p1 = ex2_approx(fmaf(hf ? x1[2 * i + 1] : x0[2 * i + 1], c, -mc));
+          for (int i = 0; i < 32; ++i) x1[i] = -INFINITY;
+        }
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub) {
+          uint32_t v[16], vr[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float p0 = ex2_approx(fmaf(sub ? x1[2 * i] : x0[2 * i], c, -mc));
+            const float p1 = ex2_approx(fmaf(sub ? x1[2 * i + 1] : x0[2 * i + 1], c, -mc));
             s4[i & 1] += p0;
             s4[2 + (i & 1)] += p1;
             v[i] = pack_bf16x2(p0, p1);
             vr[i] = pack_bf16x2_residual(p0, p1, v[i]);
           }
-          tmem_st32(tmem + lane_base + kColS + hf * 32, v);
-          tmem_st32(tmem + lane_base + kColS + 64 + hf * 32, vr);
+          tmem_st16(tmem + lane_base + col_s + sub * 16, v);
+          tmem_st16(tmem + lane_base + col_s + 32 + sub * 16, vr);
         }
       }
       const float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
@@ -346,21 +376,27 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar(BAR_P_FULL));
-      if (threadIdx.x == 64) PSA_FWD_MARK(it, 9);
+      if (threadIdx.x == 128) PSA_FWD_MARK(it, 9);
     }
 
-    // ---- epilogue: O / l -> bf16, lse
+    // ---- epilogue: O / l -> bf16, lse.  The two halves of the row sum meet in shared memory.
+    {
+      float* slot = xchg + (n_it & 1) * 2 * kTile;
+      slot[hfz * kTile + r] = l_run;
+      pair_sync();
+      l_run += slot[(hfz ^ 1) * kTile + r];
+    }
     if (n_it > 0) {
       mbar_wait(bar(BAR_O_FULL), (n_it - 1) & 1, wctx);
       tc_fence_after();
     }
     const float inv_l = 1.f / l_run;
     const int64_t row = int64_t(rec.row0) + r;
-    __nv_bfloat16* orow = prm.o + (row * prm.Hq + h) * D;
+    __nv_bfloat16* orow = prm.o + (row * prm.Hq + h) * D + hfz * (D / 2);
 #pragma unroll
-    for (int ch = 0; ch < D / 32; ++ch) {
+    for (int ch = 0; ch < D / 64; ++ch) {
       uint32_t v[32];
-      tmem_ld32_wait(tmem + lane_base + kColO + ch * 32, v);
+      tmem_ld32_wait(tmem + lane_base + kColO + hfz * (D / 2) + ch * 32, v);
       if (row_valid) {
         uint4* dst = reinterpret_cast<uint4*>(orow + ch * 32);
 #pragma unroll
@@ -374,7 +410,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
       }
     }
-    if (row_valid) {
+    if (row_valid && hfz == 0) {
       const float mc = (m_run == -INFINITY) ? 0.f : m_run * c;
       prm.lse[int64_t(h) * prm.T + row] = (mc + log2f(l_run)) * 0.6931471805599453f;
     }
