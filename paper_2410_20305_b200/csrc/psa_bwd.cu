@@ -184,7 +184,9 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
+    // The whole warp runs this loop with warp-uniform operands; one elected lane issues.
+    {
+      const uint32_t issuer = elect_one();
       constexpr uint32_t idesc_st = umma_idesc_bf16(kTile, kTile, false, false);  // K/V and Q/dO, all K-major
       constexpr uint32_t idesc_dv = umma_idesc_bf16(kTile, D, false, true);       // P^T (TMEM) x dO (MN-major)
       constexpr uint32_t idesc_dk = umma_idesc_bf16(kTile, D, false, true);       // dS^T (K-major) x Q (MN-major)
@@ -210,9 +212,9 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = ((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4;
-          umma_ss_lo(tmem + kColS, k_k + off, q_lo + off, idesc_st, kk > 0);
+          umma_ss_w(tmem + kColS, k_k + off, q_lo + off, idesc_st, kk > 0, issuer);
         }
-        umma_commit(bar(B_S_FULL));
+        umma_commit_w(bar(B_S_FULL), issuer);
       };
       issue_s(0);
       for (int it = 0; it < n_it; ++it) {
@@ -231,9 +233,9 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = ((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4;
-          umma_ss_lo(tmem + kColDP, v_k + off, do_k + off, idesc_st, kk > 0);
+          umma_ss_w(tmem + kColDP, v_k + off, do_k + off, idesc_st, kk > 0, issuer);
         }
-        umma_commit(bar(B_DP_FULL));
+        umma_commit_w(bar(B_DP_FULL), issuer);
         // dV += P^T dO   (reduction over the 128 query rows, 16 per instruction)
         mbar_wait(bar(B_P_FULL), it & 1, wctx);
         tc_fence_after();
@@ -243,10 +245,10 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         for (int term = 0; term < n_terms; ++term) {
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk)
-            umma_ts_lo(tmem + kColDV, tmem + kColS + (kk >> 2) * 64 + term * 32 + (kk & 3) * 8,
-                       do_mn + kk * (2048 >> 4), idesc_dv, (it > 0) || (kk > 0) || (term > 0));
+            umma_ts_w(tmem + kColDV, tmem + kColS + (kk >> 2) * 64 + term * 32 + (kk & 3) * 8,
+                       do_mn + kk * (2048 >> 4), idesc_dv, (it > 0) || (kk > 0) || (term > 0), issuer);
         }
-        umma_commit(bar(B_DO_EMPTY));
+        umma_commit_w(bar(B_DO_EMPTY), issuer);
         PSA_TRACE_MARK(it, 15);
         // The next S^T goes in now, so that the compute warps can start on it while the dK / dQ
         // products of this iteration run.
@@ -261,19 +263,19 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           // dQ first: the workers are waiting to read it out, and the next dP^T for them to finish.
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk)
-            umma_ss_lo(tmem + kColDP, ds_mn + kk * (2048 >> 4), k_mn + kk * (2048 >> 4), idesc_dq,
-                       (kk > 0) || (term > 0));
-          if (term + 1 == n_terms) umma_commit(bar(B_DQ_FULL));
+            umma_ss_w(tmem + kColDP, ds_mn + kk * (2048 >> 4), k_mn + kk * (2048 >> 4), idesc_dq,
+                       (kk > 0) || (term > 0), issuer);
+          if (term + 1 == n_terms) umma_commit_w(bar(B_DQ_FULL), issuer);
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk)
-            umma_ss_lo(tmem + kColDK, ds_k + (((kk >> 2) * 16384 + (kk & 3) * 32) >> 4),
-                       (st ? q1_mn : q0_mn) + kk * (2048 >> 4), idesc_dk, (it > 0) || (kk > 0) || (term > 0));
-          if (term + 1 < n_terms) umma_commit(bar(B_DS_EMPTY));
+            umma_ss_w(tmem + kColDK, ds_k + (((kk >> 2) * 16384 + (kk & 3) * 32) >> 4),
+                       (st ? q1_mn : q0_mn) + kk * (2048 >> 4), idesc_dk, (it > 0) || (kk > 0) || (term > 0), issuer);
+          if (term + 1 < n_terms) umma_commit_w(bar(B_DS_EMPTY), issuer);
         }
-        umma_commit(bar(B_Q_EMPTY0 + st));
+        umma_commit_w(bar(B_Q_EMPTY0 + st), issuer);
         PSA_TRACE_MARK(it, 4);
       }
-      umma_commit(bar(B_DONE));   // every product, the last dK included, has completed
+      umma_commit_w(bar(B_DONE), issuer);   // every product, the last dK included, has completed
     }
     __syncwarp();
   }  // warps 2, 3 of the first warpgroup are idle

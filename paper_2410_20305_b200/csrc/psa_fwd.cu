@@ -42,7 +42,7 @@ constexpr int kFwdThreads = 384;
 constexpr int kSoftmaxThreads = 256;
 // Register split of the 80 per thread the launch bound allows: the first warpgroup (producer,
 // issuer) gives registers to the two softmax warpgroups.
-constexpr int kRegsWg0 = 40, kRegsSoftmax = 96;
+constexpr int kRegsWg0 = 48, kRegsSoftmax = 96;
 constexpr uint32_t kTmemCols = 256;   // S: columns [0,128), O: columns [128, 128+D)
 constexpr uint32_t kColS = 0, kColO = 128;
 
@@ -147,7 +147,9 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __syncwarp();
    } else if (warp == 1) {
     // ------------------------------------------------------------ UMMA issuer
-    if (lane == 0) {
+    // The whole warp runs this loop with warp-uniform operands; one elected lane issues.
+    {
+      const uint32_t issuer = elect_one();
       constexpr uint32_t idesc_s = umma_idesc_bf16(kTile, kTile, false, false);  // Q, K both K-major
       constexpr uint32_t idesc_o = umma_idesc_bf16(kTile, D, false, true);       // P (TMEM), V MN-major
       // Low descriptor words (start address + LBO); the high word is a constant.
@@ -163,10 +165,10 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = ((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4;
-          umma_ss_lo(tmem + kColS, q_k + off, k_k + off, idesc_s, kk > 0);
+          umma_ss_w(tmem + kColS, q_k + off, k_k + off, idesc_s, kk > 0, issuer);
         }
-        umma_commit(bar(BAR_K_EMPTY));
-        umma_commit(bar(BAR_S_FULL));
+        umma_commit_w(bar(BAR_K_EMPTY), issuer);
+        umma_commit_w(bar(BAR_S_FULL), issuer);
         PSA_FWD_MARK(it, 2);
         mbar_wait(bar(BAR_V_FULL), it & 1, wctx);
         PSA_FWD_MARK(it, 3);
@@ -180,12 +182,12 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk) {
             // A: 16 keys of P = 8 TMEM columns (two bf16 per column).  B: 16 key rows of V.
-            umma_ts_lo(tmem + kColO, tmem + kColS + (kk >> 2) * 64 + term * 32 + (kk & 3) * 8, v_mn + kk * (2048 >> 4), idesc_o,
-                       (it > 0) || (kk > 0) || (term > 0));
+            umma_ts_w(tmem + kColO, tmem + kColS + (kk >> 2) * 64 + term * 32 + (kk & 3) * 8, v_mn + kk * (2048 >> 4), idesc_o,
+                       (it > 0) || (kk > 0) || (term > 0), issuer);
           }
         }
-        umma_commit(bar(BAR_V_EMPTY));
-        umma_commit(bar(BAR_O_FULL));
+        umma_commit_w(bar(BAR_V_EMPTY), issuer);
+        umma_commit_w(bar(BAR_O_FULL), issuer);
         PSA_FWD_MARK(it, 5);
       }
     }
