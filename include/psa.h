@@ -193,6 +193,30 @@ psa_status_t psa_bwd_static_scratch(const psa_plan_t* plan, const void* d_o, con
                                     void* stream);
 
 /*
+ * psa_step_host -- one forward and one backward pass of the attention (Algorithm 3; the
+ * two calls above) on HOST buffers.  The call enqueues on `stream`, in this order: the
+ * copies of q, k, v, d_o from host memory into the arena, psa_fwd, psa_bwd, and the copies
+ * of o, lse, dq, dk, dv back to host memory.  It does not synchronise: the outputs are valid
+ * once the stream has reached the end of the call's work.  Calls on different streams with
+ * different arenas overlap (one call's copies with another's kernels).
+ *   h_q, h_do   host bf16 [T, Hq, d]       h_k, h_v    host bf16 [T, Hkv, d]      (in)
+ *   h_o, h_dq   host bf16 [T, Hq, d]       h_dk, h_dv  host bf16 [T, Hkv, d]      (out)
+ *   h_lse       host fp32 [Hq, T]                                                (out)
+ *               Pinned (page-locked) host memory makes the copies asynchronous; pageable
+ *               memory works but serialises them with the host.
+ *   arena       device memory of at least psa_step_host_arena_bytes(plan) bytes, 256-byte
+ *               aligned, owned by the caller; it holds the device copies of every tensor
+ *               and the backward scratch.  Contents on entry are ignored, on exit undefined.
+ *               The call allocates nothing.
+ * Errors: INVALID_ARG (null pointer, arena too small), ALIGNMENT, CUDA.
+ */
+size_t psa_step_host_arena_bytes(const psa_plan_t* plan);
+psa_status_t psa_step_host(const psa_plan_t* plan, const void* h_q, const void* h_k, const void* h_v,
+                           const void* h_do, void* h_o, float* h_lse, void* h_dq, void* h_dk,
+                           void* h_dv, void* arena, size_t arena_bytes, int32_t* device_status,
+                           void* stream);
+
+/*
  * dpo_logp -- summed log-probabilities per response (Section 2.1: the total
  * log probability of each completion; Section 3.2: responses are recovered at
  * loss time from their boundaries).

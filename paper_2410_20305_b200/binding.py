@@ -25,6 +25,7 @@ EXPORTED_SYMBOLS = (
     "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
     "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp", "psa_profile_events",
     "psa_bwd_static_scratch", "dpo_loss", "dpo_logp_bwd", "psa_pack_ffd", "psa_position_ids", "psa_rope",
+    "psa_step_host_arena_bytes", "psa_step_host",
 )
 
 
@@ -70,7 +71,10 @@ def load_library():
     lib.dpo_logp_bwd.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp]
     lib.dpo_logp.argtypes = [vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     for name in EXPORTED_SYMBOLS:
-        if name != "psa_status_string":
+        if name == "psa_step_host_arena_bytes":
+            lib.psa_step_host_arena_bytes.restype = C.c_size_t
+            lib.psa_step_host_arena_bytes.argtypes = [C.c_void_p]
+        elif name != "psa_status_string":
             getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -239,6 +243,27 @@ def psa_bwd_static_scratch(plan: Plan, d_o, q, k, v, o, lse, dq, dk, dv, status=
            load_library().psa_bwd_static_scratch(plan._h, _ptr(d_o), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
                                                  _ptr(dq), _ptr(dk), _ptr(dv), _ptr(status), _stream(stream)))
     return dq, dk, dv
+
+
+def psa_step_host_arena_bytes(plan: Plan) -> int:
+    """Bytes of device memory psa_step_host needs as its arena for this plan."""
+    return int(load_library().psa_step_host_arena_bytes(plan._h))
+
+
+def psa_step_host(plan: Plan, h_q, h_k, h_v, h_do, h_o, h_lse, h_dq, h_dk, h_dv, arena, status=None, stream=None):
+    """Forward + backward on HOST tensors (pinned for asynchronous copies): enqueues the
+    copies in, psa_fwd, psa_bwd and the copies out on `stream` and returns without
+    synchronising.  `arena` is a uint8 CUDA tensor of at least psa_step_host_arena_bytes(plan)
+    bytes; nothing is allocated here."""
+    import torch
+    for t in (h_q, h_k, h_v, h_do, h_o, h_dq, h_dk, h_dv):
+        assert not t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
+    assert not h_lse.is_cuda and h_lse.dtype == torch.float32 and h_lse.is_contiguous()
+    assert arena.is_cuda and arena.dtype == torch.uint8 and arena.is_contiguous()
+    _check("psa_step_host",
+           load_library().psa_step_host(plan._h, _ptr(h_q), _ptr(h_k), _ptr(h_v), _ptr(h_do), _ptr(h_o), _ptr(h_lse),
+                                        _ptr(h_dq), _ptr(h_dk), _ptr(h_dv), _ptr(arena),
+                                        C.c_size_t(arena.numel()), _ptr(status), _stream(stream)))
 
 
 def dpo_loss(policy_logps, ref_logps, beta, stream=None):
