@@ -272,11 +272,11 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           float x[32];
           load_chunk(sub, x);
 #pragma unroll
-          for (int i = 0; i < 32; i += 4) {
-            m4[0] = fmaxf(m4[0], x[i]);
-            m4[1] = fmaxf(m4[1], x[i + 1]);
-            m4[2] = fmaxf(m4[2], x[i + 2]);
-            m4[3] = fmaxf(m4[3], x[i + 3]);
+          for (int i = 0; i < 32; i += 8) {
+            m4[0] = max3(m4[0], x[i], x[i + 1]);
+            m4[1] = max3(m4[1], x[i + 2], x[i + 3]);
+            m4[2] = max3(m4[2], x[i + 4], x[i + 5]);
+            m4[3] = max3(m4[3], x[i + 6], x[i + 7]);
           }
         }
         mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
@@ -319,6 +319,8 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (threadIdx.x == 128) PSA_FWD_MARK(it, 8);
       const float mc = (m_run == -INFINITY) ? 0.f : m_run * c;
       float s4[4] = {0.f, 0.f, 0.f, 0.f};
+      uint64_t sum2[2] = {0ull, 0ull};                 // two packed pairs of partial row sums
+      const uint64_t c2 = pack_f32x2(c, c), mc2 = pack_f32x2(-mc, -mc);
       if (!precise) {
         // P -> bf16 over the thread's own S columns: the 32 values of chunk sub go to columns
         // [16 sub, 16 sub + 16) of them, which never reaches a column that is still to be read.
@@ -333,10 +335,11 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             load_chunk(sub, x);
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              const float p0 = ex2_approx(fmaf(x[2 * i], c, -mc));
-              const float p1 = ex2_approx(fmaf(x[2 * i + 1], c, -mc));
-              s4[i & 1] += p0;
-              s4[2 + (i & 1)] += p1;
+              // two scores per instruction for the scale-and-shift and for the row sum
+              float t0, t1;
+              unpack_f32x2(fma_f32x2(pack_f32x2(x[2 * i], x[2 * i + 1]), c2, mc2), t0, t1);
+              const float p0 = ex2_approx(t0), p1 = ex2_approx(t1);
+              sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(p0, p1));
               v[i] = pack_bf16x2(p0, p1);
             }
           }
@@ -372,6 +375,13 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           tmem_st16(tmem + lane_base + col_s + sub * 16, v);
           tmem_st16(tmem + lane_base + col_s + 32 + sub * 16, vr);
         }
+      }
+      {
+        float a0, a1, b0, b1;
+        unpack_f32x2(sum2[0], a0, a1);
+        unpack_f32x2(sum2[1], b0, b1);
+        s4[0] += a0 + a1;
+        s4[2] += b0 + b1;
       }
       const float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
       l_run += sum;
