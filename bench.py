@@ -159,6 +159,7 @@ def main():
     ap.add_argument("--workload", type=int, default=1, help="1 llama3-8b, 2 long-prompt, 3 multi-turn, 4 short-many")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-layer", action="store_true")
     ap.add_argument("--no-paired", action="store_true")
     ap.add_argument("--no-logp", action="store_true", help="attention only (small footprint, for ncu captures)")
     args = ap.parse_args()
@@ -306,6 +307,53 @@ def main():
                   "ideal_pair_ratio": pplan.useful_pairs / U, "token_ratio": pp.total_tokens / T}
         del pq, pk, pv, pdo, po, plse, pws, pdq, pdk, pdv
 
+    # ---- attention-layer level (a "next" row): QKV and output projections (library GEMMs through
+    # torch.matmul), rotary embedding on the shared layout's position ids, psa_fwd / psa_bwd, and the
+    # projections' backward; the same on the paired layout.
+    layer = None
+    if not args.no_layer and rank == 0:
+        def layer_ms(pk_, seed):
+            Tl = pk_.total_tokens
+            hid = Hq * d
+            g = torch.Generator(device=dev); g.manual_seed(seed)
+            rn = lambda *shape: (torch.randn(*shape, generator=g, device=dev) * 0.02).to(torch.bfloat16)
+            x = (torch.randn(Tl, hid, generator=g, device=dev)).to(torch.bfloat16)
+            dout = (torch.randn(Tl, hid, generator=g, device=dev)).to(torch.bfloat16)
+            wq, wk, wv, wo = rn(hid, Hq * d), rn(hid, Hkv * d), rn(hid, Hkv * d), rn(Hq * d, hid)
+            pos = torch.as_tensor(B.psa_position_ids(pk_.cu_seqlens, pk_.prefix_len, pk_.chosen_len, pk_.rejected_len)).to(dev)
+            neg = -pos
+            lplan = B.psa_plan(pk_.cu_seqlens, pk_.prefix_len, pk_.chosen_len, pk_.rejected_len, Hq, Hkv, d)
+            lws = torch.empty(lplan.bwd_workspace_bytes, dtype=torch.uint8, device=dev)
+
+            def run():
+                q_ = (x @ wq).view(Tl, Hq, d); k_ = (x @ wk).view(Tl, Hkv, d); v_ = (x @ wv).view(Tl, Hkv, d)
+                B.psa_rope(q_, pos, out=q_); B.psa_rope(k_, pos, out=k_)
+                o_, lse_ = B.psa_fwd(lplan, q_, k_, v_)
+                out = o_.view(Tl, hid) @ wo                                   # noqa: F841  (the layer's output)
+                do_ = (dout @ wo.t()).view(Tl, Hq, d)
+                dwo = o_.view(Tl, hid).t() @ dout                             # noqa: F841
+                dq_, dk_, dv_ = B.psa_bwd(lplan, do_, q_, k_, v_, o_, lse_, workspace=lws)
+                B.psa_rope(dq_, neg, out=dq_); B.psa_rope(dk_, neg, out=dk_)   # gradient of a rotation: the inverse rotation
+                dq2, dk2, dv2 = dq_.view(Tl, -1), dk_.view(Tl, -1), dv_.view(Tl, -1)
+                dx = dq2 @ wq.t() + dk2 @ wk.t() + dv2 @ wv.t()               # noqa: F841
+                dwq, dwk, dwv = x.t() @ dq2, x.t() @ dk2, x.t() @ dv2         # noqa: F841
+            for _ in range(3):
+                run()
+            torch.cuda.synchronize()
+            a, b = ev(), ev()
+            a.record()
+            for _ in range(args.steps):
+                run()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / args.steps
+        l_shared = layer_ms(pack, 2200 + args.workload)
+        l_paired = layer_ms(pack.paired(), 2300 + args.workload)
+        layer = {"hidden": Hq * d, "shared_fwd_bwd_ms": l_shared, "paired_fwd_bwd_ms": l_paired,
+                 "speedup_shared_over_paired": l_paired / l_shared,
+                 "projections": "torch.matmul (cuBLAS), bf16", "rope": "psa_rope on psa_position_ids"}
+        torch.cuda.empty_cache()
+
     # ---- end to end: psa_step_host on pinned host buffers (copies in, fwd, bwd, copies out per step).
     # Two arenas on two streams, so that one step's copies out overlap the next step's copies in
     # (the link is full duplex); a step's buffers are reused only after that step has finished.
@@ -392,6 +440,7 @@ def main():
         "gpu_launches": args.steps * (4 if args.no_logp else 5),
         "paired_layout": paired,
         "next_rows": loss_bwd,
+        "attention_layer": layer,
         "paper_context": "paper reports 1.1-1.5x (1.3-1.6x with packing) end-to-end training speedups on 8xH100; context, not the target",
     }
     if e2e:

@@ -305,6 +305,21 @@ psa_status_t dpo_loss(const float* policy_logps, const float* ref_logps, int32_t
                       float* loss, float* coef, void* stream);
 
 /*
+ * simpo_loss -- the length-normalised, reference-free paired loss (SimPO; Section 1 names it
+ * beside DPO as a paired-preference method that the shared layout serves):
+ *     loss = mean over samples s of
+ *            -log sigmoid(beta * (policy[2s] / len[2s] - policy[2s+1] / len[2s+1]) - gamma).
+ *   policy_logps  device fp32 [2 * n_samples], as written by dpo_logp
+ *   lengths       device int32 [2 * n_samples]: scored tokens of each response (all >= 1)
+ *   loss          device fp32 [1] (out)
+ *   coef          device fp32 [2 * n_samples] (out): d loss / d policy_logps, ready for dpo_logp_bwd
+ * Errors: INVALID_ARG, CUDA.  A length < 1 sets PSA_DEVSTAT_BAD_SEGMENT in device_status (may be
+ * NULL) and that sample contributes nothing.
+ */
+psa_status_t simpo_loss(const float* policy_logps, const int32_t* lengths, int32_t n_samples, float beta,
+                        float gamma, float* loss, float* coef, int32_t* device_status, void* stream);
+
+/*
  * dpo_logp_bwd -- gradient of  sum_g coef[g] * out[g]  (out as written by dpo_logp) with respect
  * to the logits:  dlogits[t][v] = sum over the labels (t, y, g) scored by row t of
  *                 coef[g] * (1[v == y] - softmax(logits[t])[v]).

@@ -314,6 +314,24 @@ def dpo_loss(policy_logps, ref_logps, beta):
     return float(loss_s.mean()), coef
 
 
+def simpo_loss(policy_logps, lengths, beta, gamma):
+    """Length-normalised, reference-free variant of the paired loss (SimPO, one of the paired
+    preference methods Section 1 names as served by the same layout): mean over the n samples of
+        -log sigmoid(beta * (pol[2s] / len[2s] - pol[2s+1] / len[2s+1]) - gamma).
+    `lengths[g]` is the number of scored tokens of response g.  Returns (loss, coef) with
+    coef[g] = d loss / d policy_logps[g]."""
+    pol = np.asarray(policy_logps, dtype=np.float64)
+    ln = np.asarray(lengths, dtype=np.float64)
+    n = len(pol) // 2
+    z = float(beta) * (pol[0::2] / ln[0::2] - pol[1::2] / ln[1::2]) - float(gamma)
+    loss_s = np.maximum(-z, 0.0) + np.log1p(np.exp(-np.abs(z)))
+    sig_neg = np.exp(-np.maximum(z, 0.0)) / (1.0 + np.exp(-np.abs(z)))      # sigmoid(-z)
+    coef = np.zeros(2 * n, dtype=np.float64)
+    coef[0::2] = -float(beta) * sig_neg / (n * ln[0::2])
+    coef[1::2] = +float(beta) * sig_neg / (n * ln[1::2])
+    return float(loss_s.mean()), coef
+
+
 def dpo_logp_grad(logits, targets, segment_ids, coef, fork_rows=(), fork_targets=(), fork_segments=()):
     """d(sum_g coef[g] * out[g]) / d logits for out = dpo_logp(...): every scored (row t, label y,
     response g) contributes coef[g] * (onehot(y) - softmax(logits[t])) to row t; rows that score

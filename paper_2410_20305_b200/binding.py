@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = (
     "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
     "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp", "psa_profile_events",
     "psa_bwd_static_scratch", "dpo_loss", "dpo_logp_bwd", "psa_pack_ffd", "psa_position_ids", "psa_rope",
-    "psa_step_host_arena_bytes", "psa_step_host",
+    "psa_step_host_arena_bytes", "psa_step_host", "simpo_loss",
 )
 
 
@@ -65,6 +65,8 @@ def load_library():
     lib.psa_bwd_static_scratch.argtypes = [vp] * 12
     lib.psa_profile_events.argtypes = [i32, vp, vp]
     lib.dpo_loss.argtypes = [vp, vp, i32, f32, vp, vp, vp]
+    lib.simpo_loss.argtypes = [vp, vp, i32, f32, f32, vp, vp, vp, vp]
+    lib.psa_step_host.argtypes = [vp] * 11 + [C.c_size_t, vp, vp]
     lib.psa_pack_ffd.argtypes = [vp, i32, i32, vp, C.POINTER(i32)]
     lib.psa_position_ids.argtypes = [vp, vp, vp, vp, i32, vp]
     lib.psa_rope.argtypes = [vp, vp, vp, i64, i32, i32, f32, vp]
@@ -277,6 +279,21 @@ def dpo_loss(policy_logps, ref_logps, beta, stream=None):
     coef = torch.empty(2 * n, dtype=torch.float32, device=policy_logps.device)
     _check("dpo_loss", load_library().dpo_loss(_ptr(policy_logps), _ptr(ref_logps), n, float(beta), _ptr(loss),
                                               _ptr(coef), _stream(stream)))
+    return loss, coef
+
+
+def simpo_loss(policy_logps, lengths, beta, gamma, status=None, stream=None):
+    """policy_logps fp32 CUDA [2n], lengths int32 CUDA [2n] (scored tokens per response) ->
+    (loss fp32 [1], coef fp32 [2n]); loss = mean_s -log sigmoid(beta * (lp_c/len_c - lp_r/len_r) - gamma)."""
+    import torch
+    assert policy_logps.is_cuda and policy_logps.dtype == torch.float32 and policy_logps.is_contiguous()
+    assert lengths.is_cuda and lengths.dtype == torch.int32 and lengths.shape == policy_logps.shape
+    n = policy_logps.numel() // 2
+    loss = torch.empty(1, dtype=torch.float32, device=policy_logps.device)
+    coef = torch.empty(2 * n, dtype=torch.float32, device=policy_logps.device)
+    _check("simpo_loss", load_library().simpo_loss(_ptr(policy_logps), _ptr(lengths), n, float(beta),
+                                                  float(gamma), _ptr(loss), _ptr(coef), _ptr(status),
+                                                  _stream(stream)))
     return loss, coef
 
 

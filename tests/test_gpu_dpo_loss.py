@@ -72,3 +72,20 @@ def test_same_token_scored_twice_by_the_fork_row():
     d = B.dpo_logp_bwd(x.cuda(), _dev(targets), _dev(seg), coef, _dev(fr), _dev(ft), _dev(fs))
     want = orc.dpo_logp_grad(wl.to_f64(x), targets, seg, [0.3, -0.8], fr, ft, fs)
     assert np.abs(d.cpu().double().numpy() - want).max() <= 1e-6
+
+
+def test_simpo_loss_matches_oracle_and_feeds_the_gradient():
+    rng = np.random.default_rng(11)
+    n = 37
+    pol = rng.normal(-80, 30, size=2 * n).astype(np.float32)
+    ln = rng.integers(1, 120, size=2 * n).astype(np.int32)
+    loss, coef = B.simpo_loss(torch.tensor(pol).cuda(), torch.tensor(ln).cuda(), 2.5, 1.4)
+    rl, rc = orc.simpo_loss(pol.astype(np.float64), ln, 2.5, 1.4)
+    assert abs(loss.item() - rl) <= 1e-5 * max(1.0, abs(rl))
+    assert np.abs(coef.cpu().numpy().astype(np.float64) - rc).max() <= 1e-6 * np.abs(rc).max() + 1e-9
+    # a length below one is reported, never divided by
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ln[5] = 0
+    loss2, coef2 = B.simpo_loss(torch.tensor(pol).cuda(), torch.tensor(ln).cuda(), 2.5, 1.4, status=status)
+    assert status.item() != 0 and torch.isfinite(loss2).all() and torch.isfinite(coef2).all()
+    assert coef2[4].item() == 0.0 and coef2[5].item() == 0.0

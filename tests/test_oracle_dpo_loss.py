@@ -68,3 +68,31 @@ def test_logit_gradient_finite_differences():
     for idx in [(0, 1), (1, 4), (1, 6), (2, 3), (4, 0)]:
         zp = x.copy(); zm = x.copy(); zp[idx] += eps; zm[idx] -= eps
         assert abs((f(zp) - f(zm)) / (2 * eps) - g[idx]) < 1e-8
+
+
+def test_simpo_loss_closed_forms_and_reduction_to_dpo():
+    # equal length-normalised log-probs, gamma 0: loss = ln 2; with gamma: -log sigmoid(-gamma)
+    pol = np.array([-6.0, -9.0, -1.0, -2.0]); ln = np.array([2, 3, 5, 10])
+    loss, coef = orc.simpo_loss(pol, ln, beta=2.0, gamma=0.0)
+    assert abs(loss - np.log(2.0)) < 1e-15
+    assert np.allclose(coef, [-2.0 / (2 * 2 * 2), 2.0 / (2 * 2 * 3), -2.0 / (2 * 2 * 5), 2.0 / (2 * 2 * 10)], atol=1e-16)
+    loss, _ = orc.simpo_loss(pol, ln, beta=2.0, gamma=0.7)
+    assert abs(loss - np.log1p(np.exp(0.7))) < 1e-15
+    # unit lengths, zero reference, gamma 0: the DPO loss of Eq. 1 (pinned above on its own)
+    rng = np.random.default_rng(3)
+    pol = rng.normal(-30, 8, size=10)
+    l1, c1 = orc.simpo_loss(pol, np.ones(10), 0.4, 0.0)
+    l2, c2 = orc.dpo_loss(pol, np.zeros(10), 0.4)
+    assert abs(l1 - l2) < 1e-15 and np.allclose(c1, c2, atol=1e-16)
+
+
+def test_simpo_loss_matches_torch_autograd():
+    rng = np.random.default_rng(5)
+    pol = rng.normal(-60, 20, size=14); ln = rng.integers(1, 90, size=14)
+    tp = torch.tensor(pol, requires_grad=True)
+    tl_ = torch.tensor(ln, dtype=torch.float64)
+    z = 2.5 * (tp[0::2] / tl_[0::2] - tp[1::2] / tl_[1::2]) - 1.2
+    tl = -torch.nn.functional.logsigmoid(z).mean()
+    tl.backward()
+    loss, coef = orc.simpo_loss(pol, ln, 2.5, 1.2)
+    assert abs(loss - tl.item()) < 1e-13 and np.allclose(coef, tp.grad.numpy(), atol=1e-15)
