@@ -1,7 +1,7 @@
 // psa_bwd: exact gradient of psa_fwd under the prefix-sharing mask with packing
 // (Algorithm 3; Section 3.1).  Probabilities are recomputed from lse.
 //
-//   1. preprocess:  delta[h][t] = dO[t,h,:] . O[t,h,:]   (fp32), dq_accum = 0
+//   1. preprocess:  delta[h][t] = dO[t,h,:] . O[t,h,:]   (fp32), dq_accum = 0   (one kernel)
 //   2. main kernel: one CTA per (key tile j, kv head); it walks the query heads of the
 //      group and, for each, the live query tiles i of the transposed tile map.  All
 //      products are formed transposed (rows = keys) so that dK and dV accumulate in
@@ -557,11 +557,13 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   }
 }
 
-// delta[h][t] = sum_c dO[t,h,c] * O[t,h,c]; one 16-byte load per thread and tensor.
+// delta[h][t] = sum_c dO[t,h,c] * O[t,h,c]; one 16-byte load per thread and tensor.  The kernel also
+// clears the fp32 dq accumulator (same element mapping), which saves a separate pass over it.
 template <int D>
 __global__ void __launch_bounds__(256)
 psa_bwd_delta_kernel(const __nv_bfloat16* __restrict__ d_o, const __nv_bfloat16* __restrict__ o,
-                     float* __restrict__ delta, int64_t n_rows /* T*Hq */, int32_t T, int32_t Hq) {
+                     float* __restrict__ delta, float* __restrict__ dq_accum, int64_t n_rows /* T*Hq */, int32_t T,
+                     int32_t Hq) {
   constexpr int kLanes = D / 8;  // threads per (t, h) row
   const int64_t gid = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t row = gid / kLanes;
@@ -570,6 +572,10 @@ psa_bwd_delta_kernel(const __nv_bfloat16* __restrict__ d_o, const __nv_bfloat16*
   if (row < n_rows) {
     const uint4 a = reinterpret_cast<const uint4*>(d_o + row * D)[part];
     const uint4 b = reinterpret_cast<const uint4*>(o + row * D)[part];
+    // the same thread clears the eight accumulator elements that belong to its eight inputs
+    float4* z = reinterpret_cast<float4*>(dq_accum + row * D + part * 8);
+    z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+    z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
     const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -618,11 +624,10 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
     return PSA_ERR_CUDA;
 
   const int64_t n_rows = T * plan->Hq;
-  if (cudaMemsetAsync(dq_accum, 0, size_t(n_rows) * D * sizeof(float), stream) != cudaSuccess) return PSA_ERR_CUDA;
   {
     const int64_t threads = n_rows * (D / 8);
     psa_bwd_delta_kernel<D><<<unsigned((threads + 255) / 256), 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(d_o), static_cast<const __nv_bfloat16*>(o), delta, n_rows, plan->T,
+        static_cast<const __nv_bfloat16*>(d_o), static_cast<const __nv_bfloat16*>(o), delta, dq_accum, n_rows, plan->T,
         plan->Hq);
   }
   BwdParams prm;
