@@ -196,7 +196,7 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       // MN-major operand by 16 rows (2048 bytes).
       const uint32_t k_k = smem_desc_lo(sK, 16), v_k = smem_desc_lo(sV, 16), do_k = smem_desc_lo(sDO, 16);
       const uint32_t q0_k = smem_desc_lo(sQ(0), 16), q1_k = smem_desc_lo(sQ(1), 16);
-      const uint32_t ds_k = smem_desc_lo(sDS, 16), ds_mn = smem_desc_lo(sDS, 16384);
+      const uint32_t ds_mn = smem_desc_lo(sDS, 16384);
       const uint32_t do_mn = smem_desc_lo(sDO, L::kSubBytes), k_mn = smem_desc_lo(sK, L::kSubBytes);
       const uint32_t q0_mn = smem_desc_lo(sQ(0), L::kSubBytes), q1_mn = smem_desc_lo(sQ(1), L::kSubBytes);
       mbar_wait(bar(B_KV_FULL), 0, wctx);
@@ -253,26 +253,34 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // The next S^T goes in now, so that the compute warps can start on it while the dK / dQ
         // products of this iteration run.
         if (it + 1 < n_it) issue_s(it + 1);
-        // dK += dS^T Q ; dQ = dS K.  The two terms of a PRECISE tile pass through the one
-        // shared-memory buffer one after the other.
+        // dK += dS^T Q ; dQ = dS K.  dS^T reaches dK from TMEM (the workers leave it, as bf16 pairs
+        // and with the second term of a PRECISE tile beside it, in the columns of dP^T they have
+        // read) and dQ from the shared-memory buffer, whose two PRECISE terms pass through it one
+        // after the other.  dK goes first: dQ's accumulator overwrites those columns.
+        mbar_wait(bar(B_DS_FULL), ds_ph, wctx);
+        ds_ph ^= 1;
+        tc_fence_after();
+        PSA_TRACE_MARK(it, 3);
         for (int term = 0; term < n_terms; ++term) {
-          mbar_wait(bar(B_DS_FULL), ds_ph, wctx);
-          ds_ph ^= 1;
-          tc_fence_after();
-          PSA_TRACE_MARK(it, 3);
-          // dQ first: the workers are waiting to read it out, and the next dP^T for them to finish.
+#pragma unroll
+          for (int kk = 0; kk < kTile / 16; ++kk)
+            umma_ts_w(tmem + kColDK, tmem + kColDP + (kk >> 2) * 64 + term * 32 + (kk & 3) * 8,
+                      (st ? q1_mn : q0_mn) + kk * (2048 >> 4), idesc_dk, (it > 0) || (kk > 0) || (term > 0), issuer);
+        }
+        umma_commit_w(bar(B_Q_EMPTY0 + st), issuer);
+        for (int term = 0; term < n_terms; ++term) {
+          if (term > 0) {
+            umma_commit_w(bar(B_DS_EMPTY), issuer);
+            mbar_wait(bar(B_DS_FULL), ds_ph, wctx);
+            ds_ph ^= 1;
+            tc_fence_after();
+          }
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk)
             umma_ss_w(tmem + kColDP, ds_mn + kk * (2048 >> 4), k_mn + kk * (2048 >> 4), idesc_dq,
                        (kk > 0) || (term > 0), issuer);
-          if (term + 1 == n_terms) umma_commit_w(bar(B_DQ_FULL), issuer);
-#pragma unroll
-          for (int kk = 0; kk < kTile / 16; ++kk)
-            umma_ss_w(tmem + kColDK, ds_k + (((kk >> 2) * 16384 + (kk & 3) * 32) >> 4),
-                       (st ? q1_mn : q0_mn) + kk * (2048 >> 4), idesc_dk, (it > 0) || (kk > 0) || (term > 0), issuer);
-          if (term + 1 < n_terms) umma_commit_w(bar(B_DS_EMPTY), issuer);
         }
-        umma_commit_w(bar(B_Q_EMPTY0 + st), issuer);
+        umma_commit_w(bar(B_DQ_FULL), issuer);
         PSA_TRACE_MARK(it, 4);
       }
       umma_commit_w(bar(B_DONE), issuer);   // every product, the last dK included, has completed
@@ -437,7 +445,18 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           const uint32_t chunk = uint32_t(j * 4 + c4) ^ uint32_t(r & 7);
           st_shared_v4(row_addr + chunk * 16, w[4 * c4], w[4 * c4 + 1], w[4 * c4 + 2], w[4 * c4 + 3]);
         }
+        // The same values for dK, which takes dS^T from TMEM: over the first 32 of this thread's 64
+        // dP^T columns, all of which it has read by now (chunk 0 before the first store).
+        tmem_st16(tmem + lane_base + kColDP + half * 64 + j * 16, w);
       }
+      if constexpr (kPrecise) {
+        // second term of dS^T for dK: the other 32 of the thread's own columns
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+          tmem_st16(tmem + lane_base + kColDP + half * 64 + 32 + j * 16,
+                    reinterpret_cast<const uint32_t(&)[16]>(ds_lo[j * 16]));
+      }
+      tc_wait_st();
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(bar(B_DS_FULL));
