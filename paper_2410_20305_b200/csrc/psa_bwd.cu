@@ -16,12 +16,12 @@
 //   warp 0        TMA producer: K, V once; Q double-buffered, dO single-buffered per iteration
 //   warp 1        UMMA issuer (tcgen05, all five products); warps 2, 3 idle
 //   warps 4..11   workers: one thread per (key row, half of the 128 query columns);
-//                 P^T -> TMEM (bf16, over S^T), dS^T -> shared memory (bf16, 128-byte swizzle) for
-//                 the dK and dQ products
+//                 P^T -> TMEM (bf16, over S^T) for dV;  dS^T -> TMEM (bf16, over dP^T) for dK and
+//                 -> shared memory (bf16, 128-byte swizzle) for dQ
 //   warps 12..15  dQ drain: TMEM -> registers (columns released at once) -> shared-memory staging
 //                 -> TMA reduce-add (cp.reduce.async.bulk.tensor, fp32) into dq_accum
 // Registers are moved between the warpgroups with setmaxnreg (the drain holds a whole dQ row).
-// TMEM columns: [0,128) S^T / P^T, [128,256) dP^T / dQ, [256,256+D) dV, [384,384+D) dK.
+// TMEM columns: [0,128) S^T / P^T, [128,256) dP^T / dS^T / dQ, [256,256+D) dV, [384,384+D) dK.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
