@@ -89,10 +89,20 @@ psa_status_t psa_plan(const int32_t* cu_seqlens, const int32_t* prefix_len,
                       int32_t head_dim, float softmax_scale, int32_t flags,
                       void* stream, psa_plan_t** out);
 
-/* Copies a HOST_ONLY plan's tile map to the current device (no-op if already there). */
+/*
+ * Copies a HOST_ONLY plan's tile map to the current device (no-op if already there).  The copy is
+ * asynchronous on `stream` (from a pinned staging buffer owned by the library): kernels that use
+ * the plan must run on that stream or be ordered after it.
+ */
 psa_status_t psa_plan_upload(psa_plan_t* plan, void* stream);
 
-/* Frees the plan's host and device metadata.  NULL is accepted. */
+/*
+ * Frees the plan's host metadata and returns its device metadata (a few hundred KB) to a small
+ * cache inside the library, from which the next plan takes it: building a plan per step costs no
+ * cudaMalloc / cudaFree and does not wait for the device.  The call does not wait either: work that
+ * was enqueued with the plan may still be running; the library orders the next owner's upload
+ * behind it.  The streams the plan was used on must still exist.  NULL is accepted.
+ */
 psa_status_t psa_plan_destroy(psa_plan_t* plan);
 
 /*

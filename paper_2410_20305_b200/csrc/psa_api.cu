@@ -18,6 +18,7 @@ extern "C" psa_status_t psa_fwd(const psa_plan_t* plan, const void* q, const voi
   if (!q || !k || !v || !o || !lse) return PSA_ERR_INVALID_ARG;
   if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(o, 16) || misaligned(lse, 4))
     return PSA_ERR_ALIGNMENT;
+  psa::note_plan_use(plan, stream);
   return psa::launch_fwd(plan, q, k, v, o, lse, device_status, stream);
 }
 
@@ -32,6 +33,7 @@ extern "C" psa_status_t psa_bwd(const psa_plan_t* plan, const void* d_o, const v
       misaligned(dq, 16) || misaligned(dk, 16) || misaligned(dv, 16) || misaligned(lse, 4) ||
       misaligned(workspace, 256))
     return PSA_ERR_ALIGNMENT;
+  psa::note_plan_use(plan, stream);
   return psa::launch_bwd(plan, d_o, q, k, v, o, lse, dq, dk, dv, workspace, device_status, stream);
 }
 
@@ -70,6 +72,7 @@ extern "C" psa_status_t psa_step_host(const psa_plan_t* plan, const void* h_q, c
   const StepArena a = step_arena_layout(plan);
   if (arena_bytes < a.bytes) return PSA_ERR_INVALID_ARG;
   if (misaligned(arena, 256)) return PSA_ERR_ALIGNMENT;
+  psa::note_plan_use(plan, stream);
   char* base = static_cast<char*>(arena);
   const cudaStream_t st = cudaStream_t(stream);
   const size_t nq = size_t(plan->T) * plan->Hq * plan->d * 2, nk = size_t(plan->T) * plan->Hkv * plan->d * 2;

@@ -67,5 +67,6 @@ extern "C" psa_status_t psa_bwd_static_scratch(const psa_plan_t* plan, const voi
   if (st != PSA_OK) return st;
   // launch_bwd clears the dq accumulator itself (it must start at zero) and overwrites delta,
   // so whatever the previous call left in the array does not matter.
+  psa::note_plan_use(plan, stream);
   return psa::launch_bwd(plan, d_o, q, k, v, o, lse, dq, dk, dv, scratch, device_status, stream);
 }

@@ -34,9 +34,15 @@ struct psa_plan {
   std::vector<int32_t> fwd_entries, bwd_entries;
   // Launch order of the backward CTAs: pairs (index into kv_tiles, kv head).
   std::vector<int32_t> bwd_cta_map;
-  // device copy (one allocation)
+  // device copy (one allocation, taken from and returned to a small process-wide cache so that a
+  // plan per step costs no cudaMalloc / cudaFree and no host synchronisation)
   int device = -1;
   void* d_blob = nullptr;
+  void* h_stage = nullptr;        // pinned staging buffer the blob was uploaded from
+  size_t blob_capacity = 0;
+  void* ev_copied = nullptr;      // cudaEvent_t: the upload has left the staging buffer
+  void* ev_last_use = nullptr;    // cudaEvent_t: recorded at destroy on the streams that used the plan
+  mutable std::vector<void*> used_streams;   // streams that launched kernels reading the blob
   const psa::TileRec* d_q_tiles = nullptr;
   const psa::TileRec* d_kv_tiles = nullptr;
   const int32_t* d_fwd_entries = nullptr;
@@ -45,6 +51,13 @@ struct psa_plan {
 };
 
 namespace psa {
+// Remembers that kernels reading the plan's device blob were enqueued on `stream`.
+inline void note_plan_use(const psa_plan_t* plan, void* stream) {
+  for (void* s : plan->used_streams)
+    if (s == stream) return;
+  plan->used_streams.push_back(stream);
+}
+
 // Returns PSA_OK if no CUDA error is pending, else PSA_ERR_CUDA; with PSA_DEBUG set in the
 // environment the CUDA error string is written to stderr.
 psa_status_t check_last_cuda_error(const char* where);

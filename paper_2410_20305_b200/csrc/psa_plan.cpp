@@ -10,8 +10,10 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <numeric>
+#include <vector>
 
 #include "psa_internal.h"
 
@@ -184,6 +186,71 @@ extern "C" psa_status_t psa_plan(const int32_t* cu_seqlens, const int32_t* prefi
   return PSA_OK;
 }
 
+namespace {
+// Process-wide cache of plan blobs.  An entry is a device allocation, a pinned staging buffer of
+// the same size and two events: `copied` (the last upload has been read out of the staging buffer)
+// and `last_use` (every kernel that read the device blob under its previous owner has finished).
+struct BlobEntry {
+  int device = -1;
+  void* dptr = nullptr;
+  void* hptr = nullptr;
+  size_t capacity = 0;
+  cudaEvent_t copied = nullptr, last_use = nullptr;
+  bool last_use_valid = false;
+};
+constexpr size_t kBlobCacheMax = 16;
+std::mutex g_blob_mutex;
+std::vector<BlobEntry> g_blob_cache;
+
+void free_entry(BlobEntry& e) {
+  if (e.dptr) cudaFree(e.dptr);
+  if (e.hptr) cudaFreeHost(e.hptr);
+  if (e.copied) cudaEventDestroy(e.copied);
+  if (e.last_use) cudaEventDestroy(e.last_use);
+  e = BlobEntry{};
+}
+
+bool take_entry(int device, size_t bytes, BlobEntry* out) {
+  {
+    std::lock_guard<std::mutex> lock(g_blob_mutex);
+    int best = -1;
+    for (size_t i = 0; i < g_blob_cache.size(); ++i) {
+      const BlobEntry& e = g_blob_cache[i];
+      if (e.device == device && e.capacity >= bytes && (best < 0 || e.capacity < g_blob_cache[best].capacity))
+        best = int(i);
+    }
+    if (best >= 0) {
+      *out = g_blob_cache[best];
+      g_blob_cache.erase(g_blob_cache.begin() + best);
+      return true;
+    }
+  }
+  BlobEntry e;
+  e.device = device;
+  e.capacity = (bytes + 65535) / 65536 * 65536;   // round up so that plans of similar size share entries
+  if (cudaMalloc(&e.dptr, e.capacity) != cudaSuccess || cudaMallocHost(&e.hptr, e.capacity) != cudaSuccess ||
+      cudaEventCreateWithFlags(&e.copied, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&e.last_use, cudaEventDisableTiming) != cudaSuccess) {
+    free_entry(e);
+    return false;
+  }
+  *out = e;
+  return true;
+}
+
+void give_entry(BlobEntry e) {
+  {
+    std::lock_guard<std::mutex> lock(g_blob_mutex);
+    if (g_blob_cache.size() < kBlobCacheMax) {
+      g_blob_cache.push_back(e);
+      return;
+    }
+  }
+  if (e.last_use_valid) cudaEventSynchronize(e.last_use);
+  free_entry(e);
+}
+}  // namespace
+
 extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
   if (!p) return PSA_ERR_INVALID_ARG;
   if (p->d_blob) return PSA_OK;
@@ -195,23 +262,37 @@ extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
   const size_t b4 = up(p->bwd_cta_map.size() * sizeof(int32_t));
   const size_t total = b0 + b1 + b2 + b3 + b4 + 256;
   if (cudaGetDevice(&p->device) != cudaSuccess) return PSA_ERR_CUDA;
-  void* blob = nullptr;
-  if (cudaMalloc(&blob, total) != cudaSuccess) return PSA_ERR_CUDA;
-  // Stage in one host buffer so a single copy suffices; the copy is synchronous
-  // with respect to the host buffer because it is pageable memory.
-  std::vector<char> host(total, 0);
-  std::memcpy(host.data(), p->q_tiles.data(), p->q_tiles.size() * sizeof(TileRec));
-  std::memcpy(host.data() + b0, p->kv_tiles.data(), p->kv_tiles.size() * sizeof(TileRec));
-  std::memcpy(host.data() + b0 + b1, p->fwd_entries.data(), p->fwd_entries.size() * sizeof(int32_t));
-  std::memcpy(host.data() + b0 + b1 + b2, p->bwd_entries.data(), p->bwd_entries.size() * sizeof(int32_t));
-  std::memcpy(host.data() + b0 + b1 + b2 + b3, p->bwd_cta_map.data(), p->bwd_cta_map.size() * sizeof(int32_t));
-  if (cudaMemcpyAsync(blob, host.data(), total, cudaMemcpyHostToDevice, cudaStream_t(stream)) != cudaSuccess ||
-      cudaStreamSynchronize(cudaStream_t(stream)) != cudaSuccess) {
-    cudaFree(blob);
+  BlobEntry e;
+  if (!take_entry(p->device, total, &e)) return PSA_ERR_CUDA;
+  const cudaStream_t st = cudaStream_t(stream);
+  // The staging buffer may still be feeding the previous owner's upload (not in steady state: that
+  // copy was enqueued a whole step ago), and the device blob may still be read by the previous
+  // owner's kernels: the new upload is ordered after them on the device, without a host wait.
+  bool ok = cudaEventSynchronize(e.copied) == cudaSuccess;
+  if (ok && e.last_use_valid) ok = cudaStreamWaitEvent(st, e.last_use, 0) == cudaSuccess;
+  if (ok) {
+    char* host = static_cast<char*>(e.hptr);
+    std::memcpy(host, p->q_tiles.data(), p->q_tiles.size() * sizeof(TileRec));
+    std::memcpy(host + b0, p->kv_tiles.data(), p->kv_tiles.size() * sizeof(TileRec));
+    std::memcpy(host + b0 + b1, p->fwd_entries.data(), p->fwd_entries.size() * sizeof(int32_t));
+    std::memcpy(host + b0 + b1 + b2, p->bwd_entries.data(), p->bwd_entries.size() * sizeof(int32_t));
+    std::memcpy(host + b0 + b1 + b2 + b3, p->bwd_cta_map.data(), p->bwd_cta_map.size() * sizeof(int32_t));
+    ok = cudaMemcpyAsync(e.dptr, e.hptr, total, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+         cudaEventRecord(e.copied, st) == cudaSuccess;
+  }
+  if (!ok) {
+    cudaDeviceSynchronize();
+    free_entry(e);
     return PSA_ERR_CUDA;
   }
-  char* b = static_cast<char*>(blob);
-  p->d_blob = blob;
+  char* b = static_cast<char*>(e.dptr);
+  p->d_blob = e.dptr;
+  p->h_stage = e.hptr;
+  p->blob_capacity = e.capacity;
+  p->ev_copied = e.copied;
+  p->ev_last_use = e.last_use;
+  p->used_streams.clear();
+  p->used_streams.push_back(stream);   // the upload itself
   p->d_q_tiles = reinterpret_cast<const TileRec*>(b);
   p->d_kv_tiles = reinterpret_cast<const TileRec*>(b + b0);
   p->d_fwd_entries = reinterpret_cast<const int32_t*>(b + b0 + b1);
@@ -223,7 +304,36 @@ extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
 extern "C" psa_status_t psa_plan_destroy(psa_plan_t* p) {
   if (!p) return PSA_OK;
   psa_status_t st = PSA_OK;
-  if (p->d_blob && cudaFree(p->d_blob) != cudaSuccess) st = PSA_ERR_CUDA;
+  if (p->d_blob) {
+    // Hand the blob back.  Its next owner must not overwrite it before the kernels enqueued under
+    // this plan have run: one event, recorded in turn on every stream that used the plan (each
+    // stream first waits for the previous recording, so the last recording covers them all).
+    BlobEntry e;
+    e.device = p->device;
+    e.dptr = p->d_blob;
+    e.hptr = p->h_stage;
+    e.capacity = p->blob_capacity;
+    e.copied = cudaEvent_t(p->ev_copied);
+    e.last_use = cudaEvent_t(p->ev_last_use);
+    int cur = -1;
+    bool ok = cudaGetDevice(&cur) == cudaSuccess && (cur == p->device || cudaSetDevice(p->device) == cudaSuccess);
+    bool first = true;
+    for (void* s : p->used_streams) {
+      if (!ok) break;
+      if (!first) ok = cudaStreamWaitEvent(cudaStream_t(s), e.last_use, 0) == cudaSuccess;
+      if (ok) ok = cudaEventRecord(e.last_use, cudaStream_t(s)) == cudaSuccess;
+      first = false;
+    }
+    if (!ok) {   // a stream is gone or the context is in trouble: fall back to a full wait
+      cudaGetLastError();
+      if (cudaDeviceSynchronize() != cudaSuccess) st = PSA_ERR_CUDA;
+      e.last_use_valid = false;
+    } else {
+      e.last_use_valid = true;
+    }
+    if (cur >= 0 && cur != p->device) cudaSetDevice(cur);
+    give_entry(e);
+  }
   delete p;
   return st;
 }

@@ -77,3 +77,22 @@ def test_misaligned_pointer_is_rejected():
         B._check("psa_fwd", B.load_library().psa_fwd(plan._h, q_bad.data_ptr(), k.data_ptr(), v.data_ptr(),
                                                      q.data_ptr(), torch.empty(4, device="cuda").data_ptr(), None, None))
     assert e.value.code == 4
+
+
+def test_plans_recycle_their_device_metadata_without_racing():
+    """A destroyed plan's device blob goes to the next plan.  Destroying a plan right after
+    enqueuing work and building a different one at once must not disturb the enqueued work."""
+    packs = [wl.random_pack(90 + i, 5, 700, 8, 2, 128) for i in range(4)]
+    inputs = [wl.attention_inputs(p, 7 + i) for i, p in enumerate(packs)]
+    dev_in = [tuple(t.cuda() for t in x[:3]) for x in inputs]
+    outs = []
+    for rep in range(3):
+        for p, (q, k, v) in zip(packs, dev_in):
+            plan = device_plan(p, 0.0)
+            outs.append((p, B.psa_fwd(plan, q, k, v)))
+            plan.close()   # work still queued; the next plan takes over the same blob
+    torch.cuda.synchronize()
+    refs = {id(p): oracle_fwd(p, *x[:3], None) for p, x in zip(packs, inputs)}
+    for p, (o, lse) in outs:
+        ro, rl = refs[id(p)]
+        assert max_abs(o, ro) <= TOL_O and max_abs(lse, rl) <= TOL_LSE
