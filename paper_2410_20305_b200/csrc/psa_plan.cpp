@@ -13,6 +13,8 @@
 #include <mutex>
 #include <new>
 #include <numeric>
+#include <queue>
+#include <utility>
 #include <vector>
 
 #include "psa_internal.h"
@@ -166,13 +168,53 @@ extern "C" psa_status_t psa_plan(const int32_t* cu_seqlens, const int32_t* prefi
     std::vector<int> order(n_samples);
     std::iota(order.begin(), order.end(), 0);
     std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return work[a] > work[b]; });
-    p->bwd_cta_map.reserve(p->kv_tiles.size() * n_kv_heads * 2);
+    std::vector<std::pair<int32_t, int32_t>> ctas;   // (key tile record, kv head)
+    ctas.reserve(p->kv_tiles.size() * n_kv_heads);
+    int64_t total_work = 0;
     for (int s : order)
       for (int hk = 0; hk < n_kv_heads; ++hk)
         for (int32_t t : tiles_of[s]) {
-          p->bwd_cta_map.push_back(t);
-          p->bwd_cta_map.push_back(hk);
+          ctas.emplace_back(t, hk);
+          total_work += p->kv_tiles[t].list_cnt;
         }
+    // The grouped order can leave a ragged tail (its makespan over 148 SMs is 8 % above the mean
+    // on the Llama-3-8B-shaped pack).  Alternative: hand out the last 30 % of the work longest
+    // first.  That evens out the finish but gives up the L2 locality of the tail, so it is taken
+    // only when a list-scheduling simulation says it shortens the makespan by more than 5 %.
+    {
+      int n_sm = 148;
+      if (!(flags & PSA_PLAN_HOST_ONLY)) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+          n_sm = v;
+      }
+      auto makespan = [&](const std::vector<std::pair<int32_t, int32_t>>& order_) {
+        std::priority_queue<int64_t, std::vector<int64_t>, std::greater<int64_t>> sm;
+        for (int i = 0; i < n_sm; ++i) sm.push(0);
+        int64_t end = 0;
+        for (const auto& c : order_) {
+          const int64_t t = sm.top() + p->kv_tiles[c.first].list_cnt;
+          sm.pop();
+          sm.push(t);
+          end = std::max(end, t);
+        }
+        return end;
+      };
+      std::vector<std::pair<int32_t, int32_t>> hybrid = ctas;
+      int64_t acc = 0;
+      size_t split = 0;
+      while (split < hybrid.size() && acc * 10 < total_work * 7) acc += p->kv_tiles[hybrid[split++].first].list_cnt;
+      std::stable_sort(hybrid.begin() + split, hybrid.end(), [&](const auto& a, const auto& b) {
+        return p->kv_tiles[a.first].list_cnt > p->kv_tiles[b.first].list_cnt;
+      });
+      if (makespan(ctas) * 100 > makespan(hybrid) * 105) ctas.swap(hybrid);
+    }
+    p->bwd_cta_map.reserve(ctas.size() * 2);
+    for (const auto& c : ctas) {
+      p->bwd_cta_map.push_back(c.first);
+      p->bwd_cta_map.push_back(c.second);
+    }
   }
 
   if (!(flags & PSA_PLAN_HOST_ONLY)) {
