@@ -35,6 +35,9 @@
 namespace psa {
 #ifdef PSA_TRACE
 __device__ long long g_psa_trace[64 * 16];
+__device__ long long g_psa_cta_trace[4096 * 4];   // per CTA: start, end (globaltimer ns), SM id, iterations
+__device__ long long g_psa_cta_phase[4096 * 8];   // per CTA: globaltimer at a few points of its life
+#define PSA_CTA_PHASE(k) do { if (blockIdx.x < 4096) { unsigned long long t_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_)); g_psa_cta_phase[blockIdx.x * 8 + (k)] = (long long)t_; } } while (0)
 #endif
 namespace {
 
@@ -94,6 +97,7 @@ enum {
     if (blockIdx.x == 0 && (it) < 64) g_psa_trace[(it) * 16 + (slot)] = clock64();       \
   } while (0)
 #else
+#define PSA_CTA_PHASE(k) do {} while (0)
 #define PSA_TRACE_MARK(it, slot) do {} while (0)
 #endif
 
@@ -102,7 +106,8 @@ template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-               const __grid_constant__ CUtensorMap tm_dq, const BwdParams prm) {
+               const __grid_constant__ CUtensorMap tm_dq, const __grid_constant__ CUtensorMap tm_dk,
+               const __grid_constant__ CUtensorMap tm_dv, const BwdParams prm) {
   using L = BwdSmem<D>;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = smem_u32(smem_raw);
@@ -117,6 +122,15 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   float* s_delta = reinterpret_cast<float*>(smem_raw + L::kDelta);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef PSA_TRACE
+  if (threadIdx.x == 0 && blockIdx.x < 4096) {
+    unsigned long long t; unsigned sm;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
+    g_psa_cta_trace[blockIdx.x * 4 + 0] = (long long)t;
+    g_psa_cta_trace[blockIdx.x * 4 + 2] = sm;
+  }
+#endif
   const int tile_idx = prm.cta_map[2 * blockIdx.x];
   const int hk = prm.cta_map[2 * blockIdx.x + 1];
   const int g = prm.Hq / prm.Hkv;
@@ -137,6 +151,16 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_init(bar(i), (i == B_P_FULL || i == B_DS_FULL) ? 256 : (i == B_DQ_EMPTY ? 128 : 1));
     }
     fence_mbar_init();
+    // The K and V tiles are requested right away: their flight overlaps the TMEM allocation and
+    // the CTA-wide barrier below.
+    tma_prefetch_desc(&tm_k);
+    tma_prefetch_desc(&tm_v);
+    mbar_expect_tx(bar(B_KV_FULL), 2 * L::kTileBytes);
+    for (int s = 0; s < L::kSub; ++s) tma_load_3d(sK + s * L::kSubBytes, &tm_k, s * 64, hk, rec.row0, bar(B_KV_FULL));
+    for (int s = 0; s < L::kSub; ++s) tma_load_3d(sV + s * L::kSubBytes, &tm_v, s * 64, hk, rec.row0, bar(B_KV_FULL));
+    tma_prefetch_desc(&tm_q);
+    tma_prefetch_desc(&tm_do);
+    tma_prefetch_desc(&tm_dq);
   }
   // The list is read by every role in every iteration: keep its head in shared memory.
   if (int(threadIdx.x) < n_list && int(threadIdx.x) < L::kEntCap) s_ent[threadIdx.x] = ent[threadIdx.x];
@@ -145,6 +169,7 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  if (threadIdx.x == 0) PSA_CTA_PHASE(0);
 
   // Iteration it -> (query head of the group, entry of the list).
   auto head_of = [&](int it) { return hk * g + it / n_list; };
@@ -160,14 +185,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      tma_prefetch_desc(&tm_q);
-      tma_prefetch_desc(&tm_k);
-      tma_prefetch_desc(&tm_v);
-      tma_prefetch_desc(&tm_do);
-      tma_prefetch_desc(&tm_dq);
-      mbar_expect_tx(bar(B_KV_FULL), 2 * L::kTileBytes);
-      for (int s = 0; s < L::kSub; ++s) tma_load_3d(sK + s * L::kSubBytes, &tm_k, s * 64, hk, rec.row0, bar(B_KV_FULL));
-      for (int s = 0; s < L::kSub; ++s) tma_load_3d(sV + s * L::kSubBytes, &tm_v, s * 64, hk, rec.row0, bar(B_KV_FULL));
       for (int it = 0; it < n_it; ++it) {
         const int st = it & 1;
         const int h = head_of(it);
@@ -337,6 +354,8 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_wait(bar(B_S_FULL), it & 1, wctx);
       tc_fence_after();
       if (leader) PSA_TRACE_MARK(it, 5);
+      if (leader && it == 0) PSA_CTA_PHASE(1);
+      if (leader && it == 1) PSA_CTA_PHASE(6);
       float p[64];
       {
         uint32_t sv[64];   // both loads in flight, one wait
@@ -485,10 +504,50 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (entry_of(it) & 2) iteration(it, std::true_type{});
       else iteration(it, std::false_type{});
     }
+    if (leader) PSA_CTA_PHASE(2);
     mbar_wait(bar(B_DONE), 0, wctx);
     tc_fence_after();
+    if (leader) PSA_CTA_PHASE(3);
 
     // ---- epilogue: this half's columns of dV and dK (scaled) -> bf16
+    if (rec.len - rec.local0 >= kTile) {
+      // Full tile: rows go through shared memory (the K and V buffers are free now) in the
+      // 128-byte-swizzled layout of the tensor maps, and two TMA stores per tensor write them
+      // out coalesced.  (A ragged last tile must not touch the rows of the next sample, which the
+      // box would cover: it takes the per-thread path below.)
+#pragma unroll
+      for (int which = 0; which < 2; ++which) {
+        const float mul = which ? prm.scale : 1.f;
+        const uint32_t tile = which ? sK : sV;     // dK leaves through the K buffer, dV through V's
+#pragma unroll
+        for (int ch = 0; ch < DH / 32; ++ch) {
+          uint32_t v[32];
+          tmem_ld32_wait(tmem + lane_base + (which ? kColDK : kColDV) + half * DH + ch * 32, v);
+          // 64-column sub-tile of this thread's columns, then the 16-byte chunk inside its row
+          const int col0 = half * DH + ch * 32;
+          const uint32_t row_addr = tile + (col0 >> 6) * L::kSubBytes + r * 128;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t chunk = uint32_t(((col0 & 63) >> 3) + i) ^ uint32_t(r & 7);
+            st_shared_v4(row_addr + chunk * 16,
+                         pack_bf16x2(__uint_as_float(v[8 * i + 0]) * mul, __uint_as_float(v[8 * i + 1]) * mul),
+                         pack_bf16x2(__uint_as_float(v[8 * i + 2]) * mul, __uint_as_float(v[8 * i + 3]) * mul),
+                         pack_bf16x2(__uint_as_float(v[8 * i + 4]) * mul, __uint_as_float(v[8 * i + 5]) * mul),
+                         pack_bf16x2(__uint_as_float(v[8 * i + 6]) * mul, __uint_as_float(v[8 * i + 7]) * mul));
+          }
+        }
+      }
+      fence_proxy_async_smem();
+      named_bar_sync(1, 256);
+      if (leader) {
+        for (int s = 0; s < L::kSub; ++s) {
+          tma_store_3d(&tm_dv, sV + s * L::kSubBytes, s * 64, hk, rec.row0);
+          tma_store_3d(&tm_dk, sK + s * L::kSubBytes, s * 64, hk, rec.row0);
+        }
+        tma_commit_group();
+        tma_wait_group_read<0>();   // shared memory must outlive the stores' reads
+      }
+    } else {
     const int64_t row = int64_t(rec.row0) + r;
     __nv_bfloat16* dv_row = prm.dv + (row * prm.Hkv + hk) * D + half * DH;
     __nv_bfloat16* dk_row = prm.dk + (row * prm.Hkv + hk) * D + half * DH;
@@ -513,6 +572,7 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
         }
       }
+    }
     }
   } else {
     // ------------------------------------------------------------ dQ drain: warps 12..15, one query row per thread
@@ -565,15 +625,26 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       if (leader) PSA_TRACE_MARK(it, 10);
     }
-    if (leader) tma_wait_group<0>();   // shared memory must outlive the last reduce
+    if (leader) tma_wait_group_read<0>();   // shared memory must outlive the last reduce's reads (the adds
+                                            // themselves complete before the kernel does)
+    if (leader) PSA_CTA_PHASE(5);
   }
 
+  if (threadIdx.x == 128) PSA_CTA_PHASE(4);   // first worker: its epilogue stores are issued
   tc_fence_before();
   __syncthreads();
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem, kBwdTmemCols);
   }
+#ifdef PSA_TRACE
+  if (threadIdx.x == 0 && blockIdx.x < 4096) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    g_psa_cta_trace[blockIdx.x * 4 + 1] = (long long)t;
+    g_psa_cta_trace[blockIdx.x * 4 + 3] = n_it;
+  }
+#endif
 }
 
 // delta[h][t] = sum_c dO[t,h,c] * O[t,h,c]; one 16-byte load per thread and tensor.  The kernel also
@@ -634,10 +705,11 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
   float* dq_accum = reinterpret_cast<float*>(wsp + ws.dq_accum_off);
   float* delta = reinterpret_cast<float*>(wsp + ws.delta_off);
 
-  CUtensorMap tm_q, tm_k, tm_v, tm_do, tm_dq;
+  CUtensorMap tm_q, tm_k, tm_v, tm_do, tm_dq, tm_dk, tm_dv;
   if (!make_tile_map_bf16(&tm_q, q, T, plan->Hq, D) || !make_tile_map_bf16(&tm_k, k, T, plan->Hkv, D) ||
       !make_tile_map_bf16(&tm_v, v, T, plan->Hkv, D) || !make_tile_map_bf16(&tm_do, d_o, T, plan->Hq, D) ||
-      !make_tile_map(&tm_dq, dq_accum, T, plan->Hq, D, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, 32, 128))
+      !make_tile_map(&tm_dq, dq_accum, T, plan->Hq, D, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, 32, 128) ||
+      !make_tile_map_bf16(&tm_dk, dk, T, plan->Hkv, D) || !make_tile_map_bf16(&tm_dv, dv, T, plan->Hkv, D))
     return PSA_ERR_CUDA;
   if (cudaFuncSetAttribute(psa_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kRequest) != cudaSuccess)
     return PSA_ERR_CUDA;
@@ -667,7 +739,7 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
   const unsigned grid = unsigned(plan->kv_tiles.size()) * unsigned(plan->Hkv);
   {
     ProfileScope prof(1, stream);
-    psa_bwd_kernel<D><<<grid, kBwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_dq, prm);
+    psa_bwd_kernel<D><<<grid, kBwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_dq, tm_dk, tm_dv, prm);
   }
   {
     const int64_t n_vec4 = n_rows * D / 4;
@@ -691,6 +763,12 @@ psa_status_t launch_bwd(const psa_plan_t* plan, const void* d_o, const void* q, 
 
 #ifdef PSA_TRACE
 // Debug builds only: copies the 64 x 16 timestamp table of the last psa_bwd launch to the host.
+extern "C" int psa_trace_dump_phases(long long* host_out) {
+  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_cta_phase, sizeof(long long) * 4096 * 8));
+}
+extern "C" int psa_trace_dump_ctas(long long* host_out) {
+  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_cta_trace, sizeof(long long) * 4096 * 4));
+}
 extern "C" int psa_trace_dump(long long* host_out) {
   return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_trace, sizeof(long long) * 64 * 16));
 }
