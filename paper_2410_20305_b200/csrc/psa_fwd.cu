@@ -27,6 +27,7 @@ namespace psa {
 // Debug builds (-DPSA_TRACE) record SM-clock timestamps of the first CTA's hand-offs.
 #ifdef PSA_TRACE
 __device__ long long g_psa_trace_fwd[64 * 16];
+__device__ long long g_psa_cta_trace_fwd[8192 * 4];   // per CTA: start, end (globaltimer ns), SM id, iterations
 #define PSA_FWD_MARK(it, slot)                                                            \
   do {                                                                                    \
     if (blockIdx.x == 0 && (it) < 64) g_psa_trace_fwd[(it) * 16 + (slot)] = clock64();     \
@@ -79,7 +80,8 @@ enum { BAR_Q_FULL = 0, BAR_K_FULL, BAR_V_FULL, BAR_K_EMPTY, BAR_V_EMPTY, BAR_S_F
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 2)
 psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-               const __grid_constant__ CUtensorMap tm_v, const FwdParams prm) {
+               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+               const FwdParams prm) {
   using L = FwdSmem<D>;
   extern __shared__ uint8_t smem_raw[];
   // 128-byte-swizzled tiles need 1024-byte alignment.
@@ -92,6 +94,15 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + L::kAbort);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#ifdef PSA_TRACE
+  if (threadIdx.x == 0 && blockIdx.x < 8192) {
+    unsigned long long t; unsigned sm;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
+    g_psa_cta_trace_fwd[blockIdx.x * 4 + 0] = (long long)t;
+    g_psa_cta_trace_fwd[blockIdx.x * 4 + 2] = sm;
+  }
+#endif
   const int tile_idx = blockIdx.x / prm.Hq;
   const int h = blockIdx.x % prm.Hq;
   const int hk = h / (prm.Hq / prm.Hkv);
@@ -114,6 +125,21 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     mbar_init(bar(BAR_P_FULL), kSoftmaxThreads);
     mbar_init(bar(BAR_O_FULL), 1);
     fence_mbar_init();
+    // Q and the first K, V tiles are requested right away: their flight overlaps the TMEM
+    // allocation and the CTA-wide barrier below.  (This thread is also the producer.)
+    tma_prefetch_desc(&tm_q);
+    tma_prefetch_desc(&tm_k);
+    tma_prefetch_desc(&tm_v);
+    mbar_expect_tx(bar(BAR_Q_FULL), L::kTileBytes);
+    for (int s = 0; s < L::kSub; ++s) tma_load_3d(sQ + s * L::kSubBytes, &tm_q, s * 64, h, rec.row0, bar(BAR_Q_FULL));
+    if (n_it > 0) {
+      const int krow = rec.ds + (ent_g[0] >> 2) * kTile;
+      mbar_expect_tx(bar(BAR_K_FULL), L::kTileBytes);
+      for (int s = 0; s < L::kSub; ++s) tma_load_3d(sK + s * L::kSubBytes, &tm_k, s * 64, hk, krow, bar(BAR_K_FULL));
+      mbar_expect_tx(bar(BAR_V_FULL), L::kTileBytes);
+      for (int s = 0; s < L::kSub; ++s) tma_load_3d(sV + s * L::kSubBytes, &tm_v, s * 64, hk, krow, bar(BAR_V_FULL));
+    }
+    tma_prefetch_desc(&tm_o);
   }
   if (int(threadIdx.x) < n_it && int(threadIdx.x) < L::kEntCap) s_ent[threadIdx.x] = ent_g[threadIdx.x];
   if (warp == 0) {
@@ -129,17 +155,12 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
    if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      tma_prefetch_desc(&tm_q);
-      tma_prefetch_desc(&tm_k);
-      tma_prefetch_desc(&tm_v);
-      mbar_expect_tx(bar(BAR_Q_FULL), L::kTileBytes);
-      for (int s = 0; s < L::kSub; ++s) tma_load_3d(sQ + s * L::kSubBytes, &tm_q, s * 64, h, rec.row0, bar(BAR_Q_FULL));
-      for (int it = 0; it < n_it; ++it) {
+      for (int it = 1; it < n_it; ++it) {   // iteration 0 was requested before the CTA-wide barrier
         const int krow = rec.ds + (ent(it) >> 2) * kTile;
-        if (it > 0) mbar_wait(bar(BAR_K_EMPTY), (it - 1) & 1, wctx);
+        mbar_wait(bar(BAR_K_EMPTY), (it - 1) & 1, wctx);
         mbar_expect_tx(bar(BAR_K_FULL), L::kTileBytes);
         for (int s = 0; s < L::kSub; ++s) tma_load_3d(sK + s * L::kSubBytes, &tm_k, s * 64, hk, krow, bar(BAR_K_FULL));
-        if (it > 0) mbar_wait(bar(BAR_V_EMPTY), (it - 1) & 1, wctx);
+        mbar_wait(bar(BAR_V_EMPTY), (it - 1) & 1, wctx);
         mbar_expect_tx(bar(BAR_V_FULL), L::kTileBytes);
         for (int s = 0; s < L::kSub; ++s) tma_load_3d(sV + s * L::kSubBytes, &tm_v, s * 64, hk, krow, bar(BAR_V_FULL));
       }
@@ -405,11 +426,28 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const float inv_l = 1.f / l_run;
     const int64_t row = int64_t(rec.row0) + r;
     __nv_bfloat16* orow = prm.o + (row * prm.Hq + h) * D + hfz * (D / 2);
+    // A full tile leaves through shared memory (the Q buffer is free now) in the 128-byte-swizzled
+    // layout of the tensor map and one TMA store per 64-column sub-tile writes it out coalesced.
+    // (A ragged last tile must not touch the rows of the next sample, which the box would cover:
+    // it takes the per-thread stores.)
+    const bool full_tile = rec.len - rec.local0 >= kTile;
 #pragma unroll
     for (int ch = 0; ch < D / 64; ++ch) {
       uint32_t v[32];
       tmem_ld32_wait(tmem + lane_base + kColO + hfz * (D / 2) + ch * 32, v);
-      if (row_valid) {
+      if (full_tile) {
+        const int col0 = hfz * (D / 2) + ch * 32;
+        const uint32_t row_addr = sQ + (col0 >> 6) * L::kSubBytes + r * 128;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t chunk = uint32_t(((col0 & 63) >> 3) + i) ^ uint32_t(r & 7);
+          st_shared_v4(row_addr + chunk * 16,
+                       pack_bf16x2(__uint_as_float(v[8 * i + 0]) * inv_l, __uint_as_float(v[8 * i + 1]) * inv_l),
+                       pack_bf16x2(__uint_as_float(v[8 * i + 2]) * inv_l, __uint_as_float(v[8 * i + 3]) * inv_l),
+                       pack_bf16x2(__uint_as_float(v[8 * i + 4]) * inv_l, __uint_as_float(v[8 * i + 5]) * inv_l),
+                       pack_bf16x2(__uint_as_float(v[8 * i + 6]) * inv_l, __uint_as_float(v[8 * i + 7]) * inv_l));
+        }
+      } else if (row_valid) {
         uint4* dst = reinterpret_cast<uint4*>(orow + ch * 32);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -426,6 +464,15 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const float mc = (m_run == -INFINITY) ? 0.f : m_run * c;
       prm.lse[int64_t(h) * prm.T + row] = (mc + log2f(l_run)) * 0.6931471805599453f;
     }
+    if (full_tile) {
+      fence_proxy_async_smem();
+      asm volatile("bar.sync 5, 256;" ::: "memory");   // the eight softmax warps
+      if (threadIdx.x == 128) {
+        for (int s = 0; s < L::kSub; ++s) tma_store_3d(&tm_o, sQ + s * L::kSubBytes, s * 64, h, rec.row0);
+        tma_commit_group();
+        tma_wait_group_read<0>();   // shared memory must outlive the stores' reads
+      }
+    }
   }
 
   tc_fence_before();
@@ -434,15 +481,23 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
   }
+#ifdef PSA_TRACE
+  if (threadIdx.x == 0 && blockIdx.x < 8192) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    g_psa_cta_trace_fwd[blockIdx.x * 4 + 1] = (long long)t;
+    g_psa_cta_trace_fwd[blockIdx.x * 4 + 3] = n_it;
+  }
+#endif
 }
 
 template <int D>
 psa_status_t launch_fwd_t(const psa_plan_t* plan, const void* q, const void* k, const void* v, void* o, float* lse,
                           int32_t* device_status, cudaStream_t stream) {
   using L = FwdSmem<D>;
-  CUtensorMap tm_q, tm_k, tm_v;
+  CUtensorMap tm_q, tm_k, tm_v, tm_o;
   if (!make_tile_map_bf16(&tm_q, q, plan->T, plan->Hq, D) || !make_tile_map_bf16(&tm_k, k, plan->T, plan->Hkv, D) ||
-      !make_tile_map_bf16(&tm_v, v, plan->T, plan->Hkv, D))
+      !make_tile_map_bf16(&tm_v, v, plan->T, plan->Hkv, D) || !make_tile_map_bf16(&tm_o, o, plan->T, plan->Hq, D))
     return PSA_ERR_CUDA;
   if (cudaFuncSetAttribute(psa_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kRequest) != cudaSuccess)
     return PSA_ERR_CUDA;
@@ -459,7 +514,7 @@ psa_status_t launch_fwd_t(const psa_plan_t* plan, const void* q, const void* k, 
   const unsigned grid = unsigned(plan->q_tiles.size()) * unsigned(plan->Hq);
   {
     ProfileScope prof(0, stream);
-    psa_fwd_kernel<D><<<grid, kFwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, prm);
+    psa_fwd_kernel<D><<<grid, kFwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, tm_o, prm);
   }
   return check_last_cuda_error("psa_fwd launch");
 }
@@ -475,6 +530,9 @@ psa_status_t launch_fwd(const psa_plan_t* plan, const void* q, const void* k, co
 }  // namespace psa
 
 #ifdef PSA_TRACE
+extern "C" int psa_trace_dump_ctas_fwd(long long* host_out) {
+  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_cta_trace_fwd, sizeof(long long) * 8192 * 4));
+}
 extern "C" int psa_trace_dump_fwd(long long* host_out) {
   return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_trace_fwd, sizeof(long long) * 64 * 16));
 }
