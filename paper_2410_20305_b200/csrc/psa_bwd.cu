@@ -160,6 +160,14 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     for (int s = 0; s < L::kSub; ++s) tma_load_3d(sV + s * L::kSubBytes, &tm_v, s * 64, hk, rec.row0, bar(B_KV_FULL));
     tma_prefetch_desc(&tm_q);
     tma_prefetch_desc(&tm_do);
+    // ... and so are Q and dO of the first iteration (head hk * g, first entry of the list).
+    if (n_it > 0) {
+      const int qrow0 = rec.ds + (ent[0] >> 2) * kTile;
+      mbar_expect_tx(bar(B_Q_FULL0), L::kTileBytes);
+      for (int s = 0; s < L::kSub; ++s) tma_load_3d(sQ(0) + s * L::kSubBytes, &tm_q, s * 64, hk * g, qrow0, bar(B_Q_FULL0));
+      mbar_expect_tx(bar(B_DO_FULL), L::kTileBytes);
+      for (int s = 0; s < L::kSub; ++s) tma_load_3d(sDO + s * L::kSubBytes, &tm_do, s * 64, hk * g, qrow0, bar(B_DO_FULL));
+    }
     tma_prefetch_desc(&tm_dq);
   }
   // The list is read by every role in every iteration: keep its head in shared memory.
@@ -185,14 +193,14 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      for (int it = 0; it < n_it; ++it) {
+      for (int it = 1; it < n_it; ++it) {   // iteration 0 was requested before the CTA-wide barrier
         const int st = it & 1;
         const int h = head_of(it);
         const int qrow = rec.ds + (entry_of(it) >> 2) * kTile;
         if (it >= 2) mbar_wait(bar(B_Q_EMPTY0 + st), ((it >> 1) - 1) & 1, wctx);
         mbar_expect_tx(bar(B_Q_FULL0 + st), L::kTileBytes);
         for (int s = 0; s < L::kSub; ++s) tma_load_3d(sQ(st) + s * L::kSubBytes, &tm_q, s * 64, h, qrow, bar(B_Q_FULL0 + st));
-        if (it >= 1) mbar_wait(bar(B_DO_EMPTY), (it - 1) & 1, wctx);   // dV of the previous iteration has read dO
+        mbar_wait(bar(B_DO_EMPTY), (it - 1) & 1, wctx);   // dV of the previous iteration has read dO
         PSA_TRACE_MARK(it, 11);
         mbar_expect_tx(bar(B_DO_FULL), L::kTileBytes);
         for (int s = 0; s < L::kSub; ++s) tma_load_3d(sDO + s * L::kSubBytes, &tm_do, s * 64, h, qrow, bar(B_DO_FULL));
