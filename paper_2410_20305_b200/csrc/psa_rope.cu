@@ -18,25 +18,36 @@ namespace psa {
 namespace {
 
 constexpr int kRopeThreads = 256;
+constexpr int kRopeMaxTokens = 8;   // tokens per CTA when a token alone does not fill it
 
+// One CTA rotates `tpc` consecutive tokens (all heads): the angles of a token are computed once,
+// into shared memory, and shared by its heads; with few heads several tokens share a CTA so that
+// every thread has a 16-byte pair to work on.
 __global__ void __launch_bounds__(kRopeThreads)
 psa_rope_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
-                const int32_t* __restrict__ position_ids, int32_t H, int32_t d, float log2_theta) {
-  __shared__ float s_cos[128], s_sin[128];   // d/2 <= 128
-  const int64_t t = blockIdx.x;
+                const int32_t* __restrict__ position_ids, int64_t n_tokens, int32_t tpc, int32_t H, int32_t d,
+                float log2_theta) {
+  __shared__ float s_cos[kRopeMaxTokens * 128], s_sin[kRopeMaxTokens * 128];   // d/2 <= 128 per token
+  const int64_t t0 = int64_t(blockIdx.x) * tpc;
+  const int n_tok = int(min(int64_t(tpc), n_tokens - t0));
   const int half = d / 2;
-  const float pos = float(position_ids[t]);
-  for (int i = threadIdx.x; i < half; i += kRopeThreads) {
-    const float inv_freq = exp2f(-log2_theta * (2.0f * float(i) / float(d)));
-    sincosf(pos * inv_freq, &s_sin[i], &s_cos[i]);
+  for (int i = threadIdx.x; i < n_tok * half; i += kRopeThreads) {
+    const int tk = i / half, j = i % half;
+    const float pos = float(position_ids[t0 + tk]);
+    const float inv_freq = exp2f(-log2_theta * (2.0f * float(j) / float(d)));
+    sincosf(pos * inv_freq, &s_sin[tk * 128 + j], &s_cos[tk * 128 + j]);
   }
   __syncthreads();
   const int vec_per_half = half / 8;            // 16-byte vectors in x1 (and in x2) of one head
-  const int n_pairs = H * vec_per_half;
-  const __nv_bfloat16* xt = x + t * int64_t(H) * d;
-  __nv_bfloat16* yt = y + t * int64_t(H) * d;
+  const int pairs_per_token = H * vec_per_half;
+  const int n_pairs = n_tok * pairs_per_token;
   for (int p = threadIdx.x; p < n_pairs; p += kRopeThreads) {
-    const int h = p / vec_per_half, c = (p % vec_per_half) * 8;
+    const int tk = p / pairs_per_token, q = p % pairs_per_token;
+    const int h = q / vec_per_half, c = (q % vec_per_half) * 8;
+    const __nv_bfloat16* xt = x + (t0 + tk) * int64_t(H) * d;
+    __nv_bfloat16* yt = y + (t0 + tk) * int64_t(H) * d;
+    const float* cs = s_cos + tk * 128;
+    const float* sn = s_sin + tk * 128;
     const uint4 a = *reinterpret_cast<const uint4*>(xt + h * d + c);
     const uint4 b = *reinterpret_cast<const uint4*>(xt + h * d + half + c);
     const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
@@ -45,7 +56,7 @@ psa_rope_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__
     for (int i = 0; i < 4; ++i) {
       const float x1l = __uint_as_float(aw[i] << 16), x1h = __uint_as_float(aw[i] & 0xffff0000u);
       const float x2l = __uint_as_float(bw[i] << 16), x2h = __uint_as_float(bw[i] & 0xffff0000u);
-      const float cl = s_cos[c + 2 * i], sl = s_sin[c + 2 * i], ch = s_cos[c + 2 * i + 1], sh = s_sin[c + 2 * i + 1];
+      const float cl = cs[c + 2 * i], sl = sn[c + 2 * i], ch = cs[c + 2 * i + 1], sh = sn[c + 2 * i + 1];
       __nv_bfloat162 o1 = __floats2bfloat162_rn(x1l * cl - x2l * sl, x1h * ch - x2h * sh);
       __nv_bfloat162 o2 = __floats2bfloat162_rn(x2l * cl + x1l * sl, x2h * ch + x1h * sh);
       ow1[i] = *reinterpret_cast<uint32_t*>(&o1);
@@ -87,8 +98,12 @@ extern "C" psa_status_t psa_rope(const void* x, void* y, const int32_t* position
   if (!x || !y || !position_ids) return PSA_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(y) & 15)) return PSA_ERR_ALIGNMENT;
   if (n_tokens > 0x7fffffffLL) return PSA_ERR_UNSUPPORTED;
-  psa::psa_rope_kernel<<<unsigned(n_tokens), psa::kRopeThreads, 0, cudaStream_t(stream)>>>(
-      static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(y), position_ids, n_heads, head_dim,
-      log2f(rope_theta));
+  const int pairs_per_token = n_heads * (head_dim / 16);
+  int tpc = psa::kRopeThreads / pairs_per_token;
+  tpc = tpc < 1 ? 1 : (tpc > psa::kRopeMaxTokens ? psa::kRopeMaxTokens : tpc);
+  const int64_t grid = (n_tokens + tpc - 1) / tpc;
+  psa::psa_rope_kernel<<<unsigned(grid), psa::kRopeThreads, 0, cudaStream_t(stream)>>>(
+      static_cast<const __nv_bfloat16*>(x), static_cast<__nv_bfloat16*>(y), position_ids, n_tokens, tpc, n_heads,
+      head_dim, log2f(rope_theta));
   return psa::check_last_cuda_error("psa_rope launch");
 }
