@@ -229,6 +229,44 @@ def attention_rows(q, k, v, mask_rows, rows, softmax_scale=None):
     return o, lse
 
 
+def attention_bwd_sampled(q, k, v, d_o, o, lse, mask, rows, cols, softmax_scale=None):
+    """attention_bwd restricted to the query rows `rows` (dq) and the key positions `cols` (dk, dv),
+    for checks at sizes where the dense T x T gradient is too slow.  `o` [T, Hq, d] and `lse` [Hq, T]
+    are the results of this oracle's own forward for ALL rows (attention_fwd, or attention_rows
+    called chunk by chunk); `mask` is the dense [T, T] mask.  Same definition as attention_bwd,
+    written per row i and per column j:
+        P_ij = exp(S_ij - lse_i)   D_i = dO_i . o_i   dS_ij = P_ij (dO_i . v_j - D_i)
+        dq_i = scale sum_j dS_ij k_j      dk_j = scale sum_i dS_ij q_i      dv_j = sum_i P_ij dO_i
+    (dk, dv summed over the query heads of the kv head).  Returns
+    (dq_rows [len(rows), Hq, d], dk_cols [len(cols), Hkv, d], dv_cols [len(cols), Hkv, d])."""
+    q, k, v, d_o, o = _as_f64(q), _as_f64(k), _as_f64(v), _as_f64(d_o), _as_f64(o)
+    lse = np.asarray(lse, dtype=np.float64)
+    T, Hq, d = q.shape
+    Hkv = k.shape[1]
+    g = Hq // Hkv
+    scale = (1.0 / np.sqrt(d)) if softmax_scale is None else float(softmax_scale)
+    rows = np.asarray(rows, dtype=np.int64)
+    cols = np.asarray(cols, dtype=np.int64)
+    Dvec = (d_o * o).sum(axis=2)                       # [T, Hq]
+    dq_rows = np.zeros((len(rows), Hq, d), dtype=np.float64)
+    dk_cols = np.zeros((len(cols), Hkv, d), dtype=np.float64)
+    dv_cols = np.zeros((len(cols), Hkv, d), dtype=np.float64)
+    for h in range(Hq):
+        kh, vh, qh, doh = k[:, h // g, :], v[:, h // g, :], q[:, h, :], d_o[:, h, :]
+        # rows: everything of row i
+        S = scale * (qh[rows] @ kh.T)
+        P = np.where(mask[rows], np.exp(S - lse[h, rows][:, None]), 0.0)
+        dS = P * (doh[rows] @ vh.T - Dvec[rows, h][:, None])
+        dq_rows[:, h, :] = scale * (dS @ kh)
+        # columns: everything of key j
+        S = scale * (qh @ kh[cols].T)                   # [T, len(cols)]
+        P = np.where(mask[:, cols], np.exp(S - lse[h][:, None]), 0.0)
+        dS = P * (doh @ vh[cols].T - Dvec[:, h][:, None])
+        dk_cols[:, h // g, :] += scale * (dS.T @ qh)
+        dv_cols[:, h // g, :] += P.T @ doh
+    return dq_rows, dk_cols, dv_cols
+
+
 # --------------------------------------------------------------------------
 # Per-response summed log-probabilities
 # --------------------------------------------------------------------------

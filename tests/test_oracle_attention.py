@@ -161,3 +161,23 @@ def test_packing_is_independent_per_sample_and_rows_variant():
     rows = np.array([0, 3, pack.total_tokens - 1])
     o2, l2 = orc.attention_rows(q, k, v, mask[rows], rows)
     assert np.allclose(o2, o[rows], atol=1e-14) and np.allclose(l2, lse[:, rows], atol=1e-14)
+
+
+def test_sampled_gradient_equals_the_dense_gradient_on_its_rows_and_columns():
+    # attention_bwd_sampled is the per-row / per-column form of attention_bwd: same numbers
+    pack = wl.pack_from_lengths("s", [(70, 33, 21), (5, 0, 40), (64, 64, 0)], 4, 2, 16)
+    q, k, v, d_o = (wl.to_f64(t) for t in wl.attention_inputs(pack, 12))
+    mask = orc.packed_mask(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len)
+    o, lse = orc.attention_fwd(q, k, v, mask)
+    dq, dk, dv = orc.attention_bwd(q, k, v, d_o, mask)
+    T = pack.total_tokens
+    rows = np.array([0, 1, 69, 70, 102, 103, 123, 124, 128, 168, 169, T - 1])
+    cols = np.array([0, 5, 69, 70, 100, 110, 124, 125, 160, 232, T - 1])
+    # the forward for all rows, chunk by chunk, is the forward
+    parts = [orc.attention_rows(q, k, v, mask[r0:r0 + 50], np.arange(r0, min(T, r0 + 50))) for r0 in range(0, T, 50)]
+    o2 = np.concatenate([p[0] for p in parts], axis=0)
+    lse2 = np.concatenate([p[1] for p in parts], axis=1)
+    assert np.abs(o2 - o).max() < 1e-14 and np.abs(lse2 - lse).max() < 1e-13
+    sq, sk, sv = orc.attention_bwd_sampled(q, k, v, d_o, o2, lse2, mask, rows, cols)
+    assert np.abs(sq - dq[rows]).max() < 1e-13
+    assert np.abs(sk - dk[cols]).max() < 1e-13 and np.abs(sv - dv[cols]).max() < 1e-13
