@@ -276,6 +276,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # Planning cost on the host (build + enqueue the upload + destroy), outside the timed region.
+    t0 = time.perf_counter()
+    for _ in range(20):
+        B.psa_plan(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len, Hq, Hkv, d).close()
+    plan_host_ms = (time.perf_counter() - t0) * 1e3 / 20
+
     # Per-kernel events (the library records them right around each main kernel) are read one
     # step at a time in a separate short pass so that the timed region below stays free of syncs.
     for i in range(args.warmup):
@@ -303,7 +309,8 @@ def main():
         t_stop.record()
         sync_all()
     step_ms = t_start.elapsed_time(t_stop) / args.steps
-    att_ms = float(np.mean([e_att0[i].elapsed_time(e_att1[i]) for i in range(args.warmup, n_total)]))
+    att_all = [e_att0[i].elapsed_time(e_att1[i]) for i in range(args.warmup, n_total)]
+    att_ms = float(np.mean(att_all))
     lp_ms = float(np.mean([e_att1[i].elapsed_time(e_lp1[i]) for i in range(args.warmup, n_total)]))
     if int(status.item()) != 0:
         raise SystemExit("device status word is %d: results invalid" % int(status.item()))
@@ -465,6 +472,8 @@ def main():
                    "l2": "inputs larger than L2 (q, o, dO, dq are 133 MB each; logits %.1f GB)" % (T * VOCAB * 2 / 1e9),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "attention_fwd_bwd_ms": att_ms,
+        "attention_fwd_bwd_ms_median_min": [float(np.median(att_all)), float(np.min(att_all))],
+        "plan_ms_host": plan_host_ms,
         "pct_of_bf16_peak": {"measured": value / world / peaks["bf16_tflops"], "nominal": value / world / NOMINAL_BF16_TFLOPS,
                              "peak_source": peaks["source"]},
         "tokens_per_s": world * T / (step_ms * 1e-3),
