@@ -1,6 +1,7 @@
 // Internal definitions shared by the host planner and the kernel launchers.
 #pragma once
 #include <cstdint>
+#include <mutex>
 #include <vector>
 
 #include "psa.h"
@@ -43,6 +44,7 @@ struct psa_plan {
   void* ev_copied = nullptr;      // cudaEvent_t: the upload has left the staging buffer
   void* ev_last_use = nullptr;    // cudaEvent_t: recorded at destroy on the streams that used the plan
   mutable std::vector<void*> used_streams;   // streams that launched kernels reading the blob
+  mutable std::mutex used_mutex;             // launches from several host threads may share a plan
   const psa::TileRec* d_q_tiles = nullptr;
   const psa::TileRec* d_kv_tiles = nullptr;
   const int32_t* d_fwd_entries = nullptr;
@@ -53,6 +55,7 @@ struct psa_plan {
 namespace psa {
 // Remembers that kernels reading the plan's device blob were enqueued on `stream`.
 inline void note_plan_use(const psa_plan_t* plan, void* stream) {
+  std::lock_guard<std::mutex> lock(plan->used_mutex);
   for (void* s : plan->used_streams)
     if (s == stream) return;
   plan->used_streams.push_back(stream);
