@@ -287,6 +287,18 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       float mx;
       {
         float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
+        if (cls == 0u) {
+          // nothing masked (every FULL tile): both chunks with one wait
+          uint32_t v[64];
+          tmem_ld64_wait(tmem + lane_base + col_s, v);
+#pragma unroll
+          for (int i = 0; i < 64; i += 8) {
+            m4[0] = max3(m4[0], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+            m4[1] = max3(m4[1], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+            m4[2] = max3(m4[2], __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+            m4[3] = max3(m4[3], __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+          }
+        } else
 #pragma unroll
         for (int sub = 0; sub < 2; ++sub) {
           if (chunk_class(sub) == 2u) continue;
