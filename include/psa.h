@@ -330,6 +330,17 @@ psa_status_t simpo_loss(const float* policy_logps, const int32_t* lengths, int32
                         float gamma, float* loss, float* coef, int32_t* device_status, void* stream);
 
 /*
+ * orpo_loss -- the odds-ratio paired loss (ORPO; Section 1 names it beside DPO and SimPO): with
+ * a_g = policy[g] / len[g], P_g = exp(a_g) and lo_g = a_g - log(1 - P_g),
+ *     loss = mean over samples s of  -a_{2s} + lambda * -log sigmoid(lo_{2s} - lo_{2s+1}).
+ *   policy_logps, lengths, loss, coef, device_status   as for simpo_loss
+ * Errors: INVALID_ARG, CUDA.  A length < 1 sets PSA_DEVSTAT_BAD_SEGMENT and that sample contributes
+ * nothing.  A mean log-prob of exactly 0 (probability 1) makes the odds infinite, as in the definition.
+ */
+psa_status_t orpo_loss(const float* policy_logps, const int32_t* lengths, int32_t n_samples, float lambda,
+                       float* loss, float* coef, int32_t* device_status, void* stream);
+
+/*
  * dpo_logp_bwd -- gradient of  sum_g coef[g] * out[g]  (out as written by dpo_logp) with respect
  * to the logits:  dlogits[t][v] = sum over the labels (t, y, g) scored by row t of
  *                 coef[g] * (1[v == y] - softmax(logits[t])[v]).

@@ -370,6 +370,30 @@ def simpo_loss(policy_logps, lengths, beta, gamma):
     return float(loss_s.mean()), coef
 
 
+def orpo_loss(policy_logps, lengths, lam):
+    """Odds-ratio variant of the paired loss (ORPO, named in Section 1 beside DPO and SimPO): with
+    a_g = pol[g] / len[g] (mean token log-prob, < 0), P_g = exp(a_g) and log-odds
+    lo_g = a_g - log(1 - P_g), mean over the n samples of
+        -a_{2s}  +  lam * -log sigmoid(lo_{2s} - lo_{2s+1})
+    (the first term is the supervised loss on the chosen response).  Returns (loss, coef) with
+    coef[g] = d loss / d policy_logps[g]."""
+    pol = np.asarray(policy_logps, dtype=np.float64)
+    ln = np.asarray(lengths, dtype=np.float64)
+    n = len(pol) // 2
+    a = pol / ln
+    one_minus_p = -np.expm1(a)                          # 1 - exp(a), accurate near a = 0
+    lo = a - np.log(one_minus_p)
+    z = lo[0::2] - lo[1::2]
+    nls = np.maximum(-z, 0.0) + np.log1p(np.exp(-np.abs(z)))             # -log sigmoid(z)
+    sig_neg = np.exp(-np.maximum(z, 0.0)) / (1.0 + np.exp(-np.abs(z)))   # sigmoid(-z)
+    loss = float((-a[0::2] + float(lam) * nls).mean())
+    dlo_da = 1.0 / one_minus_p                          # d lo / d a
+    coef = np.zeros(2 * n, dtype=np.float64)
+    coef[0::2] = (-1.0 - float(lam) * sig_neg * dlo_da[0::2]) / (n * ln[0::2])
+    coef[1::2] = (+float(lam) * sig_neg * dlo_da[1::2]) / (n * ln[1::2])
+    return loss, coef
+
+
 def dpo_logp_grad(logits, targets, segment_ids, coef, fork_rows=(), fork_targets=(), fork_segments=()):
     """d(sum_g coef[g] * out[g]) / d logits for out = dpo_logp(...): every scored (row t, label y,
     response g) contributes coef[g] * (onehot(y) - softmax(logits[t])) to row t; rows that score

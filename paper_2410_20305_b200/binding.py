@@ -25,7 +25,7 @@ EXPORTED_SYMBOLS = (
     "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
     "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp", "psa_profile_events",
     "psa_bwd_static_scratch", "dpo_loss", "dpo_logp_bwd", "psa_pack_ffd", "psa_position_ids", "psa_rope",
-    "psa_step_host_arena_bytes", "psa_step_host", "simpo_loss",
+    "psa_step_host_arena_bytes", "psa_step_host", "simpo_loss", "orpo_loss",
 )
 
 
@@ -66,6 +66,7 @@ def load_library():
     lib.psa_profile_events.argtypes = [i32, vp, vp]
     lib.dpo_loss.argtypes = [vp, vp, i32, f32, vp, vp, vp]
     lib.simpo_loss.argtypes = [vp, vp, i32, f32, f32, vp, vp, vp, vp]
+    lib.orpo_loss.argtypes = [vp, vp, i32, f32, vp, vp, vp, vp]
     lib.psa_step_host.argtypes = [vp] * 11 + [C.c_size_t, vp, vp]
     lib.psa_pack_ffd.argtypes = [vp, i32, i32, vp, C.POINTER(i32)]
     lib.psa_position_ids.argtypes = [vp, vp, vp, vp, i32, vp]
@@ -294,6 +295,20 @@ def simpo_loss(policy_logps, lengths, beta, gamma, status=None, stream=None):
     _check("simpo_loss", load_library().simpo_loss(_ptr(policy_logps), _ptr(lengths), n, float(beta),
                                                   float(gamma), _ptr(loss), _ptr(coef), _ptr(status),
                                                   _stream(stream)))
+    return loss, coef
+
+
+def orpo_loss(policy_logps, lengths, lam, status=None, stream=None):
+    """policy_logps fp32 CUDA [2n], lengths int32 CUDA [2n] -> (loss fp32 [1], coef fp32 [2n]);
+    loss = mean_s  -lp_c/len_c + lam * -log sigmoid(log odds ratio of the mean-token likelihoods)."""
+    import torch
+    assert policy_logps.is_cuda and policy_logps.dtype == torch.float32 and policy_logps.is_contiguous()
+    assert lengths.is_cuda and lengths.dtype == torch.int32 and lengths.shape == policy_logps.shape
+    n = policy_logps.numel() // 2
+    loss = torch.empty(1, dtype=torch.float32, device=policy_logps.device)
+    coef = torch.empty(2 * n, dtype=torch.float32, device=policy_logps.device)
+    _check("orpo_loss", load_library().orpo_loss(_ptr(policy_logps), _ptr(lengths), n, float(lam), _ptr(loss),
+                                                _ptr(coef), _ptr(status), _stream(stream)))
     return loss, coef
 
 

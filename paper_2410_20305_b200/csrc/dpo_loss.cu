@@ -1,4 +1,4 @@
-// dpo_loss / simpo_loss / dpo_logp_bwd: the DPO loss of Eq. 1 (Section 2.1; the printed ratio of logs is
+// dpo_loss / simpo_loss / orpo_loss / dpo_logp_bwd: the DPO loss of Eq. 1 (Section 2.1; the printed ratio of logs is
 // read as  -log sigmoid(beta * [(lp_theta(c) - lp_ref(c)) - (lp_theta(r) - lp_ref(r))]),
 // averaged over the samples) and its gradient back into the logits,
 //     dlogits[t][v] = sum over labels (t, y, g) scored by row t of  coef[g] * (1[v == y] - softmax(logits[t])[v]).
@@ -147,6 +147,38 @@ __global__ void simpo_loss_kernel(const float* __restrict__ pol, const int32_t* 
   }
 }
 
+// Odds-ratio variant (ORPO); one block.
+__global__ void orpo_loss_kernel(const float* __restrict__ pol, const int32_t* __restrict__ len, int n, float lam,
+                                 float* __restrict__ loss, float* __restrict__ coef, int32_t* __restrict__ status) {
+  __shared__ float part[32];
+  float acc = 0.f;
+  for (int s = threadIdx.x; s < n; s += blockDim.x) {
+    const int lc = len[2 * s], lr = len[2 * s + 1];
+    if (lc < 1 || lr < 1) {
+      if (status) atomicOr(status, PSA_DEVSTAT_BAD_SEGMENT);
+      coef[2 * s] = 0.f;
+      coef[2 * s + 1] = 0.f;
+      continue;
+    }
+    const float ac = pol[2 * s] / float(lc), ar = pol[2 * s + 1] / float(lr);
+    const float qc = -expm1f(ac), qr = -expm1f(ar);          // 1 - P
+    const float z = (ac - logf(qc)) - (ar - logf(qr));       // log odds ratio
+    const float e = expf(-fabsf(z));
+    acc += -ac + lam * (fmaxf(-z, 0.f) + log1pf(e));
+    const float sig_neg = expf(-fmaxf(z, 0.f)) / (1.f + e);   // sigmoid(-z)
+    coef[2 * s] = (-1.f - lam * sig_neg / qc) / (float(n) * float(lc));
+    coef[2 * s + 1] = (lam * sig_neg / qr) / (float(n) * float(lr));
+  }
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float t = threadIdx.x < (blockDim.x >> 5) ? part[threadIdx.x] : 0.f;
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if (threadIdx.x == 0) *loss = n > 0 ? t / float(n) : 0.f;
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kBwdLogpThreads, 1)
 dpo_logp_bwd_kernel(const T* __restrict__ logits, int64_t vocab, int64_t row_stride, const int32_t* __restrict__ targets,
@@ -270,6 +302,14 @@ extern "C" psa_status_t simpo_loss(const float* policy_logps, const int32_t* len
   psa::simpo_loss_kernel<<<1, 256, 0, cudaStream_t(stream)>>>(policy_logps, lengths, n_samples, beta, gamma, loss, coef,
                                                              device_status);
   return psa::check_last_cuda_error("simpo_loss launch");
+}
+
+extern "C" psa_status_t orpo_loss(const float* policy_logps, const int32_t* lengths, int32_t n_samples, float lambda,
+                                  float* loss, float* coef, int32_t* device_status, void* stream) {
+  if (n_samples < 0 || !loss || (n_samples > 0 && (!policy_logps || !lengths || !coef))) return PSA_ERR_INVALID_ARG;
+  psa::orpo_loss_kernel<<<1, 256, 0, cudaStream_t(stream)>>>(policy_logps, lengths, n_samples, lambda, loss, coef,
+                                                            device_status);
+  return psa::check_last_cuda_error("orpo_loss launch");
 }
 
 extern "C" psa_status_t dpo_logp_bwd(const void* logits, int32_t logits_dtype, int64_t n_rows, int64_t vocab,

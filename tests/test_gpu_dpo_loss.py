@@ -89,3 +89,14 @@ def test_simpo_loss_matches_oracle_and_feeds_the_gradient():
     loss2, coef2 = B.simpo_loss(torch.tensor(pol).cuda(), torch.tensor(ln).cuda(), 2.5, 1.4, status=status)
     assert status.item() != 0 and torch.isfinite(loss2).all() and torch.isfinite(coef2).all()
     assert coef2[4].item() == 0.0 and coef2[5].item() == 0.0
+
+
+def test_orpo_loss_matches_oracle():
+    rng = np.random.default_rng(13)
+    n = 41
+    ln = rng.integers(2, 200, size=2 * n).astype(np.int32)
+    pol = (-rng.uniform(0.05, 4.0, size=2 * n) * ln).astype(np.float32)
+    loss, coef = B.orpo_loss(torch.tensor(pol).cuda(), torch.tensor(ln).cuda(), 0.3)
+    rl, rc = orc.orpo_loss(pol.astype(np.float64), ln, 0.3)
+    assert abs(loss.item() - rl) <= 1e-5 * max(1.0, abs(rl))
+    assert np.abs(coef.cpu().numpy().astype(np.float64) - rc).max() <= 2e-5 * np.abs(rc).max()

@@ -96,3 +96,19 @@ def test_simpo_loss_matches_torch_autograd():
     tl.backward()
     loss, coef = orc.simpo_loss(pol, ln, 2.5, 1.2)
     assert abs(loss - tl.item()) < 1e-13 and np.allclose(coef, tp.grad.numpy(), atol=1e-15)
+
+
+def test_orpo_loss_closed_form_and_torch_autograd():
+    # equal mean log-probs: the odds ratio is 1, loss = -a + lam * ln 2
+    loss, _ = orc.orpo_loss([-6.0, -9.0], [3, 4.5], 0.25)
+    assert abs(loss - (2.0 + 0.25 * np.log(2.0))) < 1e-14
+    rng = np.random.default_rng(8)
+    ln = rng.integers(2, 60, size=16)
+    pol = -rng.uniform(0.05, 3.0, size=16) * ln
+    tp = torch.tensor(pol, requires_grad=True)
+    a = tp / torch.tensor(ln, dtype=torch.float64)
+    lo = a - torch.log1p(-torch.exp(a))
+    tl = (-a[0::2] - 0.7 * torch.nn.functional.logsigmoid(lo[0::2] - lo[1::2])).mean()
+    tl.backward()
+    loss, coef = orc.orpo_loss(pol, ln, 0.7)
+    assert abs(loss - tl.item()) < 1e-12 and np.allclose(coef, tp.grad.numpy(), rtol=1e-11, atol=1e-14)
