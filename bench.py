@@ -405,6 +405,20 @@ def main():
                  "projections": "torch.matmul (cuBLAS), bf16", "rope": "psa_rope on psa_position_ids"}
         torch.cuda.empty_cache()
 
+    # ---- packing (a "next" row, host only): first-fit-decreasing over 2000 units of the workload's
+    # length distribution, shared units (P + C + R) against paired units (2P + C + R)
+    packing = None
+    if rank == 0:
+        lens, cap = wl.sample_lengths(args.workload, 2000, 3000 + args.workload)
+        shared = [p + c + r for p, c, r in lens]
+        paired_u = [min(2 * p + c + r, cap) for p, c, r in lens]   # (a unit longer than a pack would be truncated)
+        t0 = time.perf_counter()
+        _, nb_s = B.psa_pack_ffd(shared, cap)
+        _, nb_p = B.psa_pack_ffd(paired_u, cap)
+        packing = {"units": len(lens), "pack_len": cap, "packs_shared": nb_s, "packs_paired": nb_p,
+                   "packs_ratio_paired_over_shared": nb_p / nb_s, "fill_shared": sum(shared) / (nb_s * cap),
+                   "fill_paired": sum(paired_u) / (nb_p * cap), "ms_both": (time.perf_counter() - t0) * 1e3}
+
     # ---- end to end: psa_step_host on pinned host buffers (copies in, fwd, bwd, copies out per step).
     # Two arenas on two streams, so that one step's copies out overlap the next step's copies in
     # (the link is full duplex); a step's buffers are reused only after that step has finished.
@@ -494,6 +508,7 @@ def main():
         "paired_layout": paired,
         "next_rows": loss_bwd,
         "attention_layer": layer,
+        "packing": packing,
         "paper_context": "paper reports 1.1-1.5x (1.3-1.6x with packing) end-to-end training speedups on 8xH100; context, not the target",
     }
     if e2e:

@@ -78,12 +78,8 @@ def _fill(rng, draw, pack_len):
 CONFIG_NAMES = ("tiny", "llama3-8b", "long-prompt", "multi-turn", "short-many")
 
 
-def config_pack(index: int, seed: int | None = None) -> Pack:
-    """Workload `index` (0..4).  Lengths are drawn from
-    numpy.random.default_rng(1000 + index) unless a seed is given."""
-    rng = np.random.default_rng(1000 + index if seed is None else seed)
-    if index == 0:
-        return pack_from_lengths("tiny", [(256, 64, 96), (128, 80, 48)], 4, 4, 64)
+def _length_recipe(index: int):
+    """(draw, pack_len) of workload 1..4: draw(rng) -> (P, C, R)."""
     if index == 1:
         draw = lambda g: (_lognormal_clipped(g, 600, 1.0, 64, 4096),
                           _lognormal_clipped(g, 250, 1.0, 16, 1024),
@@ -99,8 +95,25 @@ def config_pack(index: int, seed: int | None = None) -> Pack:
         draw = lambda g: (int(g.integers(64, 257)), int(g.integers(64, 257)), int(g.integers(64, 257)))
         pack_len = 8192
     else:
-        raise ValueError("config index 0..4")
+        raise ValueError("config index 1..4")
+    return draw, pack_len
+
+
+def config_pack(index: int, seed: int | None = None) -> Pack:
+    """Workload `index` (0..4).  Lengths are drawn from
+    numpy.random.default_rng(1000 + index) unless a seed is given."""
+    rng = np.random.default_rng(1000 + index if seed is None else seed)
+    if index == 0:
+        return pack_from_lengths("tiny", [(256, 64, 96), (128, 80, 48)], 4, 4, 64)
+    draw, pack_len = _length_recipe(index)
     return pack_from_lengths(CONFIG_NAMES[index], _fill(rng, draw, pack_len), 32, 8, 128, pack_len)
+
+
+def sample_lengths(index: int, n: int, seed: int):
+    """n samples (P, C, R) of workload 1..4's length distribution, and its pack length."""
+    draw, pack_len = _length_recipe(index)
+    rng = np.random.default_rng(seed)
+    return [draw(rng) for _ in range(n)], pack_len
 
 
 def random_pack(seed, n_samples, max_len, n_q_heads, n_kv_heads, head_dim, allow_zero=True) -> Pack:
