@@ -488,6 +488,7 @@ def main():
         "attention_fwd_bwd_ms": att_ms,
         "attention_fwd_bwd_ms_median_min": [float(np.median(att_all)), float(np.min(att_all))],
         "plan_ms_host": plan_host_ms,
+        "plan_ms_host_per_layer_of_32": plan_host_ms / 32,   # one plan serves every layer of a step
         "pct_of_bf16_peak": {"measured": value / world / peaks["bf16_tflops"], "nominal": value / world / NOMINAL_BF16_TFLOPS,
                              "peak_source": peaks["source"]},
         "tokens_per_s": world * T / (step_ms * 1e-3),
