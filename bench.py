@@ -35,7 +35,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) of one psa_bwd_kernel launch, from the ncu capture summarised in
 # profiles/psa_bwd_kernel_llama3-8b.md (workload 1); other workloads have no capture.
-NCU_BWD_TRAFFIC_BYTES = {1: 1480.8e6}
+NCU_BWD_TRAFFIC_BYTES = {1: 1454.7e6}
 
 
 def measured_peaks():
