@@ -35,6 +35,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) of one psa_bwd_kernel launch, from the ncu capture summarised in
 # profiles/psa_bwd_kernel_llama3-8b.md (workload 1); other workloads have no capture.
+N_E2E = int(os.environ.get("PSA_BENCH_E2E_STREAMS", "3"))   # arenas / streams of the end-to-end leg
 NCU_BWD_TRAFFIC_BYTES = {1: 1454.7e6}
 
 
@@ -420,24 +421,25 @@ def main():
                    "fill_paired": sum(paired_u) / (nb_p * cap), "ms_both": (time.perf_counter() - t0) * 1e3}
 
     # ---- end to end: psa_step_host on pinned host buffers (copies in, fwd, bwd, copies out per step).
-    # Two arenas on two streams, so that one step's copies out overlap the next step's copies in
+    # A few arenas, each on a stream of its own, so that one step's copies out overlap the next step's copies in
     # (the link is full duplex); a step's buffers are reused only after that step has finished.
     e2e = None
     if not args.no_e2e:
         hq, hk, hv, hdo = (t.cpu().pin_memory() for t in (q, k, v, d_o))
-        h_out = [[torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in (o, lse, dq, dk, dv)] for _ in range(2)]
+        h_out = [[torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in (o, lse, dq, dk, dv)] for _ in range(N_E2E)]
         h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv, hdo))
         d2h = sum(t.numel() * t.element_size() for t in h_out[0])
         arena_bytes = B.psa_step_host_arena_bytes(plan0)
-        arenas = [torch.empty(arena_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
-        streams = [torch.cuda.Stream(device=dev) for _ in range(2)]
+        arenas = [torch.empty(arena_bytes, dtype=torch.uint8, device=dev) for _ in range(N_E2E)]
+        streams = [torch.cuda.Stream(device=dev) for _ in range(N_E2E)]
         plans = []   # kept alive: freeing a plan's device blob would synchronise the device mid-pipeline
 
         def e2e_run(n):
             for i in range(n):
-                s = i & 1
+                s = i % N_E2E
                 streams[s].synchronize()
-                p = B.psa_plan(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len, Hq, Hkv, d)
+                p = B.psa_plan(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len, Hq, Hkv, d,
+                               stream=streams[s].cuda_stream)
                 plans.append(p)
                 ho = h_out[s]
                 B.psa_step_host(p, hq, hk, hv, hdo, ho[0], ho[1], ho[2], ho[3], ho[4], arenas[s],
@@ -455,12 +457,12 @@ def main():
         plans.clear()
         # the last step's gradients, as read back on the host, must be the device path's
         # (dk is accumulated in a fixed order, hence bit-identical; dq's fp32 adds are not ordered)
-        last = h_out[(n_e2e - 1) & 1]
+        last = h_out[(n_e2e - 1) % N_E2E]
         assert torch.equal(last[3], dk.cpu()), "psa_step_host: dk differs from psa_bwd"
         assert (last[2].float() - dq.cpu().float()).abs().max().item() <= 0.0625, "psa_step_host: dq differs"
         e2e = {"value": (flops_fwd + flops_bwd) / e2e_ms / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "call": "psa_step_host, 2 arenas on 2 streams", "steps": n_e2e}
+               "call": "psa_step_host, %d arenas on %d streams" % (N_E2E, N_E2E), "steps": n_e2e}
         del arenas
 
     # ---- max over ranks (replicas): whole-job value = sum of the replicas' useful flops / slowest time

@@ -91,8 +91,8 @@ psa_status_t psa_plan(const int32_t* cu_seqlens, const int32_t* prefix_len,
 
 /*
  * Copies a HOST_ONLY plan's tile map to the current device (no-op if already there).  The copy is
- * asynchronous on `stream` (from a pinned staging buffer owned by the library): kernels that use
- * the plan must run on that stream or be ordered after it.
+ * asynchronous on `stream` (from a pinned staging buffer owned by the library).  Calls that use the
+ * plan on another stream make that stream wait for the copy themselves.
  */
 psa_status_t psa_plan_upload(psa_plan_t* plan, void* stream);
 

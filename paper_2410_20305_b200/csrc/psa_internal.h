@@ -53,13 +53,10 @@ struct psa_plan {
 };
 
 namespace psa {
-// Remembers that kernels reading the plan's device blob were enqueued on `stream`.
-inline void note_plan_use(const psa_plan_t* plan, void* stream) {
-  std::lock_guard<std::mutex> lock(plan->used_mutex);
-  for (void* s : plan->used_streams)
-    if (s == stream) return;
-  plan->used_streams.push_back(stream);
-}
+// Called before kernels that read the plan's device blob are enqueued on `stream`: remembers the
+// stream (psa_plan_destroy orders the blob's next owner behind it) and, the first time a stream
+// other than the upload's is used, makes it wait for the upload (which is asynchronous).
+void note_plan_use(const psa_plan_t* plan, void* stream);
 
 // Returns PSA_OK if no CUDA error is pending, else PSA_ERR_CUDA; with PSA_DEBUG set in the
 // environment the CUDA error string is written to stderr.

@@ -343,6 +343,17 @@ extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
   return PSA_OK;
 }
 
+namespace psa {
+void note_plan_use(const psa_plan_t* plan, void* stream) {
+  std::lock_guard<std::mutex> lock(plan->used_mutex);
+  for (void* s : plan->used_streams)
+    if (s == stream) return;
+  // used_streams[0] is the upload's stream; any other stream has to see the uploaded blob first
+  if (plan->ev_copied) cudaStreamWaitEvent(cudaStream_t(stream), cudaEvent_t(plan->ev_copied), 0);
+  plan->used_streams.push_back(stream);
+}
+}  // namespace psa
+
 extern "C" psa_status_t psa_plan_destroy(psa_plan_t* p) {
   if (!p) return PSA_OK;
   psa_status_t st = PSA_OK;

@@ -96,3 +96,24 @@ def test_plans_recycle_their_device_metadata_without_racing():
     for p, (o, lse) in outs:
         ro, rl = refs[id(p)]
         assert max_abs(o, ro) <= TOL_O and max_abs(lse, rl) <= TOL_LSE
+
+
+def test_plan_uploaded_on_one_stream_is_usable_on_another_at_once():
+    """The plan's upload is asynchronous on the stream given to psa_plan.  A call on a different
+    (non-blocking) stream right afterwards must order itself behind that upload, even when the
+    upload's stream is busy."""
+    pack = wl.random_pack(123, 4, 600, 8, 2, 128)
+    q, k, v, _ = wl.attention_inputs(pack, 5)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    ro, rl = oracle_fwd(pack, q, k, v, None)
+    side = torch.cuda.Stream()
+    a = torch.randn(8192, 8192, device="cuda")
+    torch.cuda.synchronize()
+    for _ in range(3):
+        b = a @ a                       # keeps the current stream busy for a while
+        plan = device_plan(pack, 0.0)   # upload queued behind it on the current stream
+        o, lse = B.psa_fwd(plan, qd, kd, vd, stream=side.cuda_stream)
+        side.synchronize()
+        assert max_abs(o, ro) <= TOL_O and max_abs(lse, rl) <= TOL_LSE
+        del b
+    torch.cuda.synchronize()
