@@ -124,7 +124,9 @@ class ClockSampler:
         if self.source == "nvml":
             reasons = [n for n in self.NAMES if self.mask & self.BITS[n]]
             return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_min_mhz": min(self.sm) if self.sm else None,
-                    "sm_max_mhz": self.max_sm, "reasons": reasons, "samples": len(self.sm), "source": "nvml, every 2 ms"}
+                    "sm_max_mhz": self.max_sm, "reasons": reasons, "samples": len(self.sm), "source": "nvml, every 2 ms",
+                    "note": "NVML's reading; inside the attention kernels ncu's sm__cycles_elapsed.avg.per_second is "
+                            "1.59-1.68 GHz (see profiles/), with no clock-event reason raised"}
         sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
         mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
         reasons = [n for i, n in enumerate(self.NAMES) if any(len(r) >= 6 and r[2 + i] == "Active" for r in self.rows)]
