@@ -1,7 +1,10 @@
 // psa_bwd: exact gradient of psa_fwd under the prefix-sharing mask with packing
 // (Algorithm 3; Section 3.1).  Probabilities are recomputed from lse.
 //
-//   1. preprocess:  delta[h][t] = dO[t,h,:] . O[t,h,:]   (fp32), dq_accum = 0   (one kernel)
+//   1. preprocess:  delta[h][t] = dO[t,h,:] . O[t,h,:]   (fp32), dq_accum = 0   (one kernel);
+//      then, only for a pack that holds rejected rows with fewer than 32 visible keys outside
+//      their sample's first query tile (prompts shorter than 32 tokens), a small kernel that
+//      recomputes delta of those rows exactly
 //   2. main kernel: one CTA per (key tile j, kv head); it walks the query heads of the
 //      group and, for each, the live query tiles i of the transposed tile map.  All
 //      products are formed transposed (rows = keys) so that dK and dV accumulate in
@@ -690,6 +693,52 @@ psa_bwd_delta_kernel(const __nv_bfloat16* __restrict__ d_o, const __nv_bfloat16*
   }
 }
 
+// Exact delta for the rejected rows of short-prompt samples that see fewer than kFewKeys keys and
+// lie outside their sample's first query tile (the main kernel recomputes delta of first-tile
+// rows itself):  delta_i = sum_j P_ij dP_ij  over the row's visible keys, P_ij = exp(scale q_i.k_j
+// - lse_i), dP_ij = dO_i.v_j, in fp32.  For such rows delta = dO.O taken from the bf16-rounded O is
+// the largest error left in dQ and dK.  One warp per (row, query head), one key per lane.
+template <int D>
+__global__ void __launch_bounds__(128)
+psa_bwd_delta_few_keys_kernel(const FewKeyRow* __restrict__ rows, const __nv_bfloat16* __restrict__ q,
+                              const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+                              const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ lse,
+                              float* __restrict__ delta, int32_t T, int32_t Hq, int32_t Hkv, float scale_log2) {
+  const FewKeyRow rec = rows[blockIdx.x];
+  const int h = blockIdx.y * 4 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (h >= Hq) return;
+  const int hk = h / (Hq / Hkv);
+  const int n_keys = rec.n_prompt + (rec.row - rec.rs_row + 1);   // < kFewKeys = 32
+  float term = 0.f;
+  if (lane < n_keys) {
+    const int64_t key = lane < rec.n_prompt ? rec.ds + lane : rec.rs_row + (lane - rec.n_prompt);
+    const uint4* q4 = reinterpret_cast<const uint4*>(q + (int64_t(rec.row) * Hq + h) * D);
+    const uint4* g4 = reinterpret_cast<const uint4*>(d_o + (int64_t(rec.row) * Hq + h) * D);
+    const uint4* k4 = reinterpret_cast<const uint4*>(k + (key * Hkv + hk) * D);
+    const uint4* v4 = reinterpret_cast<const uint4*>(v + (key * Hkv + hk) * D);
+    float s = 0.f, dp = 0.f;
+    auto dot8 = [](const uint4& a, const uint4& b, float acc) {
+      const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        acc = fmaf(__uint_as_float(aw[i] << 16), __uint_as_float(bw[i] << 16), acc);
+        acc = fmaf(__uint_as_float(aw[i] & 0xffff0000u), __uint_as_float(bw[i] & 0xffff0000u), acc);
+      }
+      return acc;
+    };
+#pragma unroll 4
+    for (int c = 0; c < D / 8; ++c) {
+      s = dot8(q4[c], k4[c], s);
+      dp = dot8(g4[c], v4[c], dp);
+    }
+    term = ex2_approx(fmaf(s, scale_log2, -lse[int64_t(h) * T + rec.row] * kLog2e)) * dp;
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) term += __shfl_xor_sync(0xffffffffu, term, off);
+  if (lane == 0) delta[int64_t(h) * T + rec.row] = term;
+}
+
 __global__ void __launch_bounds__(256)
 psa_bwd_convert_kernel(const float4* __restrict__ acc, uint2* __restrict__ dq, int64_t n_vec4) {
   const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -729,6 +778,11 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
         static_cast<const __nv_bfloat16*>(d_o), static_cast<const __nv_bfloat16*>(o), delta, dq_accum, n_rows, plan->T,
         plan->Hq);
   }
+  if (!plan->few_key_rows.empty())
+    psa_bwd_delta_few_keys_kernel<D><<<dim3(unsigned(plan->few_key_rows.size()), unsigned((plan->Hq + 3) / 4)), 128, 0, stream>>>(
+        plan->d_few_key_rows, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
+        static_cast<const __nv_bfloat16*>(v), static_cast<const __nv_bfloat16*>(d_o), lse, delta, plan->T, plan->Hq,
+        plan->Hkv, plan->scale * kLog2e);
   BwdParams prm;
   prm.tiles = plan->d_kv_tiles;
   prm.entries = plan->d_bwd_entries;

@@ -24,6 +24,18 @@ struct TileRec {
 };
 static_assert(sizeof(TileRec) == 32, "TileRec is 8 int32");
 
+// A rejected-response row that lies outside its sample's first query tile and sees fewer than
+// kFewKeys keys (a sample with a very short prompt).  Its visible keys are the packed rows
+// [ds, ds + n_prompt) and [rs_row, row].  The backward pass recomputes delta of these rows exactly.
+constexpr int kFewKeys = 32;
+struct FewKeyRow {
+  int32_t row;       // packed-row index of the query row
+  int32_t ds;        // packed-row index of the sample's first token
+  int32_t n_prompt;  // prompt length P
+  int32_t rs_row;    // packed-row index of the first rejected token
+};
+static_assert(sizeof(FewKeyRow) == 16, "FewKeyRow is 4 int32");
+
 }  // namespace psa
 
 struct psa_plan {
@@ -35,6 +47,7 @@ struct psa_plan {
   std::vector<int32_t> fwd_entries, bwd_entries;
   // Launch order of the backward CTAs: pairs (index into kv_tiles, kv head).
   std::vector<int32_t> bwd_cta_map;
+  std::vector<psa::FewKeyRow> few_key_rows;
   // device copy (one allocation, taken from and returned to a small process-wide cache so that a
   // plan per step costs no cudaMalloc / cudaFree and no host synchronisation)
   int device = -1;
@@ -50,6 +63,7 @@ struct psa_plan {
   const int32_t* d_fwd_entries = nullptr;
   const int32_t* d_bwd_entries = nullptr;
   const int32_t* d_bwd_cta_map = nullptr;
+  const psa::FewKeyRow* d_few_key_rows = nullptr;
 };
 
 namespace psa {

@@ -142,6 +142,10 @@ extern "C" psa_status_t psa_plan(const int32_t* cu_seqlens, const int32_t* prefi
       }
       p->kv_tiles.push_back(r);
     }
+    // Rejected rows past the first query tile that see fewer than kFewKeys keys (only a sample
+    // with a prompt shorter than that has any).
+    for (int q = std::max(rs, kTile); q < len && P + (q - rs + 1) < psa::kFewKeys; ++q)
+      p->few_key_rows.push_back(psa::FewKeyRow{ds + q, ds, P, ds + rs});
   }
   // Longest list first: the hardware hands out CTAs in index order, so the long
   // work items start early and the short ones fill the tail.
@@ -302,7 +306,8 @@ extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
   const size_t b2 = up(p->fwd_entries.size() * sizeof(int32_t));
   const size_t b3 = up(p->bwd_entries.size() * sizeof(int32_t));
   const size_t b4 = up(p->bwd_cta_map.size() * sizeof(int32_t));
-  const size_t total = b0 + b1 + b2 + b3 + b4 + 256;
+  const size_t b5 = up(p->few_key_rows.size() * sizeof(psa::FewKeyRow));
+  const size_t total = b0 + b1 + b2 + b3 + b4 + b5 + 256;
   if (cudaGetDevice(&p->device) != cudaSuccess) return PSA_ERR_CUDA;
   BlobEntry e;
   if (!take_entry(p->device, total, &e)) return PSA_ERR_CUDA;
@@ -319,6 +324,7 @@ extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
     std::memcpy(host + b0 + b1, p->fwd_entries.data(), p->fwd_entries.size() * sizeof(int32_t));
     std::memcpy(host + b0 + b1 + b2, p->bwd_entries.data(), p->bwd_entries.size() * sizeof(int32_t));
     std::memcpy(host + b0 + b1 + b2 + b3, p->bwd_cta_map.data(), p->bwd_cta_map.size() * sizeof(int32_t));
+    std::memcpy(host + b0 + b1 + b2 + b3 + b4, p->few_key_rows.data(), p->few_key_rows.size() * sizeof(psa::FewKeyRow));
     ok = cudaMemcpyAsync(e.dptr, e.hptr, total, cudaMemcpyHostToDevice, st) == cudaSuccess &&
          cudaEventRecord(e.copied, st) == cudaSuccess;
   }
@@ -340,6 +346,7 @@ extern "C" psa_status_t psa_plan_upload(psa_plan_t* p, void* stream) {
   p->d_fwd_entries = reinterpret_cast<const int32_t*>(b + b0 + b1);
   p->d_bwd_entries = reinterpret_cast<const int32_t*>(b + b0 + b1 + b2);
   p->d_bwd_cta_map = reinterpret_cast<const int32_t*>(b + b0 + b1 + b2 + b3);
+  p->d_few_key_rows = reinterpret_cast<const psa::FewKeyRow*>(b + b0 + b1 + b2 + b3 + b4);
   return PSA_OK;
 }
 
