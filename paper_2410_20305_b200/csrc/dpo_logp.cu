@@ -176,7 +176,8 @@ extern "C" psa_status_t dpo_logp(const void* logits, int32_t logits_dtype, int64
   if (logits_dtype != PSA_DTYPE_F32 && logits_dtype != PSA_DTYPE_BF16) return PSA_ERR_INVALID_ARG;
   if (n_rows > 0x7fffffffLL) return PSA_ERR_UNSUPPORTED;
   const int64_t esz = logits_dtype == PSA_DTYPE_F32 ? 4 : 2;
-  if ((reinterpret_cast<uintptr_t>(logits) & 15) || ((row_stride * esz) & 15)) return PSA_ERR_ALIGNMENT;
+  // the stride is not used when there is a single row
+  if ((reinterpret_cast<uintptr_t>(logits) & 15) || (n_rows > 1 && ((row_stride * esz) & 15))) return PSA_ERR_ALIGNMENT;
   cudaStream_t st = cudaStream_t(stream);
   if (n_segments > 0 && cudaMemsetAsync(out, 0, sizeof(float) * size_t(n_segments), st) != cudaSuccess)
     return PSA_ERR_CUDA;

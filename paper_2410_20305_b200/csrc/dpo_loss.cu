@@ -325,7 +325,7 @@ extern "C" psa_status_t dpo_logp_bwd(const void* logits, int32_t logits_dtype, i
   if (n_rows > 0x7fffffffLL) return PSA_ERR_UNSUPPORTED;
   const int64_t esz = logits_dtype == PSA_DTYPE_F32 ? 4 : 2;
   if ((reinterpret_cast<uintptr_t>(logits) & 15) || (reinterpret_cast<uintptr_t>(dlogits) & 15) ||
-      ((row_stride * esz) & 15))
+      (n_rows > 1 && ((row_stride * esz) & 15)))   // the stride is not used when there is a single row
     return PSA_ERR_ALIGNMENT;
   if (n_rows == 0) return PSA_OK;
   cudaStream_t st = cudaStream_t(stream);

@@ -83,3 +83,19 @@ def test_zero_rows_and_zero_segments():
     e = torch.empty(0, dtype=torch.int32, device="cuda")
     out = B.dpo_logp(x, e, e, 3)
     assert (out.cpu() == 0).all()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("vocab", [1, 3, 7, 129])
+def test_single_row_of_any_width(vocab, dtype):
+    """One row has no stride, so a vocabulary that is not a multiple of 16 bytes is accepted; the
+    ragged tail of the row is handled by scalar loads."""
+    x, tok = wl.logits_and_tokens(1, vocab, 11, 2.0, dtype)
+    seg = np.zeros(1, dtype=np.int32)
+    coef = torch.tensor([0.75], dtype=torch.float32, device="cuda")
+    out = B.dpo_logp(x.cuda(), tok.cuda(), _dev(seg), 1)
+    want = orc.dpo_logp(wl.to_f64(x), tok.numpy(), seg, 1)
+    assert abs(out.item() - want[0]) <= TOL_LOGP * max(1.0, abs(want[0]))
+    grad = B.dpo_logp_bwd(x.cuda(), tok.cuda(), _dev(seg), coef)
+    ref = orc.dpo_logp_grad(wl.to_f64(x), tok.numpy(), seg, [0.75])
+    assert np.abs(grad.cpu().double().numpy() - ref).max() <= (2e-6 if dtype == torch.float32 else 2.0 ** -8)
