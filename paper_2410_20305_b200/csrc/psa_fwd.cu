@@ -32,8 +32,18 @@ __device__ long long g_psa_cta_trace_fwd[8192 * 4];   // per CTA: start, end (gl
   do {                                                                                    \
     if (blockIdx.x == 0 && (it) < 64) g_psa_trace_fwd[(it) * 16 + (slot)] = clock64();     \
   } while (0)
+__device__ long long g_psa_cta_phase_fwd[8192 * 8];   // per CTA: globaltimer at eight points of its life
+#define PSA_FWD_PHASE(slot)                                                               \
+  do {                                                                                    \
+    if (blockIdx.x < 8192) {                                                              \
+      unsigned long long t_;                                                              \
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                               \
+      g_psa_cta_phase_fwd[blockIdx.x * 8 + (slot)] = (long long)t_;                       \
+    }                                                                                     \
+  } while (0)
 #else
 #define PSA_FWD_MARK(it, slot) do {} while (0)
+#define PSA_FWD_PHASE(slot) do {} while (0)
 #endif
 namespace {
 
@@ -149,6 +159,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  if (threadIdx.x == 128) PSA_FWD_PHASE(1);
 
   if (warp < 4) {
    setmaxnreg_dec<kRegsWg0>();
@@ -245,6 +256,8 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_wait(bar(BAR_S_FULL), it & 1, wctx);
       tc_fence_after();
       if (threadIdx.x == 128) PSA_FWD_MARK(it, 6);
+      if (threadIdx.x == 128 && it == 0) PSA_FWD_PHASE(2);
+      if (threadIdx.x == 128 && it == 1) PSA_FWD_PHASE(3);
       // Allowed keys of this row in a PARTIAL tile, relative to the tile: [0, a) and [b, b + span).
       int a = kTile, b = 0;
       uint32_t span = 0;
@@ -284,6 +297,80 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           for (int i = 0; i < 32; ++i) x[i] = __uint_as_float(v[i]);
         }
       };
+      // Fast path (every tile but the first of a list and the PRECISE ones): one pass.  The
+      // exponentials are taken against the running maximum while the tile's own maximum is
+      // found on the side; P stays in registers until the two threads of the row have agreed
+      // that the running maximum still holds (it nearly always does, see the 2^8 rule below).
+      // If it does not, nothing has been written yet and the two-pass path below redoes the tile.
+      bool fast_done = false;
+      if (it > 0 && !precise) {
+        uint32_t pk[32];
+        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        uint64_t sum2[2] = {0ull, 0ull};
+        const float mc0 = (m_run == -INFINITY) ? 0.f : m_run * c;
+        const uint64_t c2 = pack_f32x2(c, c), mc2 = pack_f32x2(-mc0, -mc0);
+        // 16 columns at a time: P of the whole tile (32 registers) has to stay live next to them
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          const uint32_t cc = chunk_class(ch >> 1);
+          if (cc == 2u) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pk[8 * ch + i] = 0u;
+            continue;
+          }
+          uint32_t v[16];
+          tmem_ld16_wait(tmem + lane_base + col_s + ch * 16, v);
+          float x[16];
+          if (cc == 1u) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const int col = hfz * 64 + ch * 16 + i;
+              const bool ok = (col < a) || (uint32_t(col - b) < span);
+              x[i] = ok ? __uint_as_float(v[i]) : -INFINITY;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) x[i] = __uint_as_float(v[i]);
+          }
+#pragma unroll
+          for (int i = 0; i < 16; i += 8) {
+            m4[0] = max3(m4[0], x[i], x[i + 1]);
+            m4[1] = max3(m4[1], x[i + 2], x[i + 3]);
+            m4[2] = max3(m4[2], x[i + 4], x[i + 5]);
+            m4[3] = max3(m4[3], x[i + 6], x[i + 7]);
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            float t0, t1;
+            unpack_f32x2(fma_f32x2(pack_f32x2(x[2 * i], x[2 * i + 1]), c2, mc2), t0, t1);
+            const float p0 = ex2_approx(t0), p1 = ex2_approx(t1);
+            sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(p0, p1));
+            pk[8 * ch + i] = pack_bf16x2(p0, p1);
+          }
+        }
+        float mxf = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        {
+          float* slot = xchg + (it & 1) * 2 * kTile;
+          slot[hfz * kTile + r] = mxf;
+          pair_sync();
+          mxf = fmaxf(mxf, slot[(hfz ^ 1) * kTile + r]);
+        }
+        const bool grow_f = (fmaxf(m_run, mxf) - m_run) * c > 8.0f;
+        if (!__any_sync(0xffffffffu, grow_f)) {
+          // the 16 values of chunk ch go to columns [8 ch, 8 ch + 8) of the thread's own 64
+          tmem_st32(tmem + lane_base + col_s, pk);
+          float a0, a1, b0, b1;
+          unpack_f32x2(sum2[0], a0, a1);
+          unpack_f32x2(sum2[1], b0, b1);
+          l_run += (a0 + a1) + (b0 + b1);
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar(BAR_P_FULL));
+          if (threadIdx.x == 128) PSA_FWD_MARK(it, 9);
+          fast_done = true;
+        }
+      }
+      if (fast_done) continue;
       float mx;
       {
         float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
@@ -424,6 +511,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (threadIdx.x == 128) PSA_FWD_MARK(it, 9);
     }
 
+    if (threadIdx.x == 128) PSA_FWD_PHASE(4);
     // ---- epilogue: O / l -> bf16, lse.  The two halves of the row sum meet in shared memory.
     {
       float* slot = xchg + (n_it & 1) * 2 * kTile;
@@ -435,6 +523,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_wait(bar(BAR_O_FULL), (n_it - 1) & 1, wctx);
       tc_fence_after();
     }
+    if (threadIdx.x == 128) PSA_FWD_PHASE(5);
     const float inv_l = 1.f / l_run;
     const int64_t row = int64_t(rec.row0) + r;
     __nv_bfloat16* orow = prm.o + (row * prm.Hq + h) * D + hfz * (D / 2);
@@ -485,6 +574,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         tma_wait_group_read<0>();   // shared memory must outlive the stores' reads
       }
     }
+    if (threadIdx.x == 128) PSA_FWD_PHASE(6);
   }
 
   tc_fence_before();
@@ -544,6 +634,9 @@ psa_status_t launch_fwd(const psa_plan_t* plan, const void* q, const void* k, co
 #ifdef PSA_TRACE
 extern "C" int psa_trace_dump_ctas_fwd(long long* host_out) {
   return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_cta_trace_fwd, sizeof(long long) * 8192 * 4));
+}
+extern "C" int psa_trace_dump_phases_fwd(long long* host_out) {
+  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_cta_phase_fwd, sizeof(long long) * 8192 * 8));
 }
 extern "C" int psa_trace_dump_fwd(long long* host_out) {
   return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_trace_fwd, sizeof(long long) * 64 * 16));
