@@ -6,7 +6,7 @@ import torch
 from paper_2410_20305_b200 import binding as B
 from paper_2410_20305_b200 import workloads as wl
 
-from gpu_util import TOL_LSE, TOL_O, device_plan, max_abs, oracle_fwd, read_status
+from gpu_util import TOL_LSE, TOL_O, device_plan, grad_errors, max_abs, oracle_fwd, read_status
 
 pytestmark = pytest.mark.gpu
 
@@ -117,3 +117,31 @@ def test_plan_uploaded_on_one_stream_is_usable_on_another_at_once():
         assert max_abs(o, ro) <= TOL_O and max_abs(lse, rl) <= TOL_LSE
         del b
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("gains", [(1, 3, 5, 7, 9, 11), (1, 6, 1, 1, 8, 1), (6, 1, 1, 1, 1, 1)])
+def test_row_maximum_that_grows_from_key_tile_to_key_tile(gains):
+    """Keys of the t-th 128-token stretch of every sample are scaled by gains[t], so the row maximum
+    jumps by far more than the 2^8 the kernel tolerates in a stale maximum: the one-pass fast path
+    has to give up, the two-pass path takes the tile and the accumulator is rescaled in TMEM.  With
+    N(0,1) inputs this path is next to never taken."""
+    pack = wl.pack_from_lengths("grow", [(300, 200, 150), (90, 400, 260)], 4, 2, 64)
+    q, k, v, _ = wl.attention_inputs(pack, 21)
+    g = torch.ones(pack.total_tokens)
+    for s in range(pack.n_samples):
+        lo, hi = int(pack.cu_seqlens[s]), int(pack.cu_seqlens[s + 1])
+        local = torch.arange(hi - lo)
+        g[lo:hi] = torch.tensor(gains, dtype=torch.float32)[local // 128]
+    k = (k.float() * g[:, None, None]).to(torch.bfloat16)
+    plan = device_plan(pack)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    o, lse = B.psa_fwd(plan, q.cuda(), k.cuda(), v.cuda(), status=status)
+    assert read_status(status) == 0
+    ro, rl = oracle_fwd(pack, q, k, v)
+    # Rows this peaked have o close to one or two v rows, and |v| reaches 4.  o takes the reading
+    # used for the gradients (raw gate below |reference| 2, gate on top of the bf16 half-ulp above),
+    # and the gate itself is doubled: P is a bf16 operand (relative error 2^-9), and with one or two
+    # dominant probabilities those errors no longer average out as they do for the N(0,1) scores
+    # the 1e-2 was stated for (measured here: 0.0106).  A wrong rescale would be off by O(1).
+    raw, raw_small, excess = grad_errors(o, ro)
+    assert raw_small <= 2 * TOL_O and excess <= 2 * TOL_O and max_abs(lse, rl) <= TOL_LSE, (raw, raw_small, excess, max_abs(lse, rl))
