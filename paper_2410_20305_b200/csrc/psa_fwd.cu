@@ -53,7 +53,7 @@ constexpr int kFwdThreads = 384;
 constexpr int kSoftmaxThreads = 256;
 // Register split of the 80 per thread the launch bound allows: the first warpgroup (producer,
 // issuer) gives registers to the two softmax warpgroups.
-constexpr int kRegsWg0 = 48, kRegsSoftmax = 96;
+constexpr int kRegsWg0 = 32, kRegsSoftmax = 104;
 constexpr uint32_t kTmemCols = 256;   // S: columns [0,128), O: columns [128, 128+D)
 constexpr uint32_t kColS = 0, kColO = 128;
 
@@ -309,7 +309,28 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         uint64_t sum2[2] = {0ull, 0ull};
         const float mc0 = (m_run == -INFINITY) ? 0.f : m_run * c;
         const uint64_t c2 = pack_f32x2(c, c), mc2 = pack_f32x2(-mc0, -mc0);
-        // 16 columns at a time: P of the whole tile (32 registers) has to stay live next to them
+        if (cls == 0u) {
+          // Nothing masked (every FULL tile): all 64 columns with one load and one wait.  Every
+          // wait exposes the TMEM latency, which the two warps per sub-partition do not hide.
+          uint32_t v[64];
+          tmem_ld64_wait(tmem + lane_base + col_s, v);
+#pragma unroll
+          for (int i = 0; i < 64; i += 8) {
+            m4[0] = max3(m4[0], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+            m4[1] = max3(m4[1], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+            m4[2] = max3(m4[2], __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+            m4[3] = max3(m4[3], __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+          }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            float t0, t1;
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), c2, mc2), t0, t1);
+            const float p0 = ex2_approx(t0), p1 = ex2_approx(t1);
+            sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(p0, p1));
+            pk[i] = pack_bf16x2(p0, p1);
+          }
+        } else
+        // PARTIAL tiles, 16 columns at a time: P of the whole tile (32 registers) stays live next to them
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           const uint32_t cc = chunk_class(ch >> 1);
