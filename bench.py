@@ -201,7 +201,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="psa", choices=["psa", "reference"])
     ap.add_argument("--workload", type=int, default=1, help="1 llama3-8b, 2 long-prompt, 3 multi-turn, 4 short-many")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -338,6 +338,24 @@ def main():
         loss_bwd = {"dpo_loss": float(loss_t.item()), "dpo_logp_bwd_ms": lb_ms, "dpo_logp_bwd_gbs": lb_bytes / lb_ms / 1e6,
                     "algorithmic_bytes": lb_bytes}
         del dlogits
+
+    # ---- the gather with every row scored (a longer stream: T x V x 2 bytes), timed alone
+    all_rows = None
+    if not args.no_logp and rank == 0:
+        seg_all = torch.from_numpy((np.arange(T) % n_seg).astype(np.int32)).to(dev)
+        for _ in range(2):
+            B.dpo_logp(logits, targets, seg_all, n_seg, out=logp.clone(), status=status)
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        scratch = torch.empty_like(logp)
+        a.record()
+        for _ in range(5):
+            B.dpo_logp(logits, targets, seg_all, n_seg, out=scratch, status=status)
+        b.record()
+        torch.cuda.synchronize()
+        ar_ms = a.elapsed_time(b) / 5
+        ar_bytes = T * (VOCAB * 2 + 8)
+        all_rows = {"rows": T, "ms": ar_ms, "gbs": ar_bytes / ar_ms / 1e6, "algorithmic_bytes": ar_bytes}
 
     # ---- the same kernels on the unshared paired layout (2n causal sequences)
     paired = None
@@ -476,6 +494,8 @@ def main():
         return
 
     peaks = measured_peaks()
+    if all_rows:
+        all_rows["frac_of_hbm"] = {"measured": all_rows["gbs"] / peaks["hbm_gbs"], "nominal": all_rows["gbs"] / NOMINAL_HBM_GBS}
     value = whole_job_tflops(flops_fwd + flops_bwd, world, att_ms)
     bwd_ms, fwd_ms, klp_ms = (float(np.mean(kernel_ms[n])) for n in ("bwd", "fwd", "logp"))
     bwd_tflops = flops_bwd / bwd_ms / 1e9
@@ -511,6 +531,7 @@ def main():
         "clocks": clocks.summary(),
         "gpu_launches": args.steps * (4 if args.no_logp else 5),
         "paired_layout": paired,
+        "dpo_logp_all_rows": all_rows,
         "next_rows": loss_bwd,
         "attention_layer": layer,
         "packing": packing,
