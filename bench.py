@@ -497,6 +497,7 @@ def main():
     if all_rows:
         all_rows["frac_of_hbm"] = {"measured": all_rows["gbs"] / peaks["hbm_gbs"], "nominal": all_rows["gbs"] / NOMINAL_HBM_GBS}
     value = whole_job_tflops(flops_fwd + flops_bwd, world, att_ms)
+    att_min_bytes = T * (6 * Hq + 6 * Hkv) * d * 2
     bwd_ms, fwd_ms, klp_ms = (float(np.mean(kernel_ms[n])) for n in ("bwd", "fwd", "logp"))
     bwd_tflops = flops_bwd / bwd_ms / 1e9
     logp_bytes = live_rows * VOCAB * 2 + 8 * live_rows + 4 * n_seg
@@ -515,6 +516,11 @@ def main():
         "plan_ms_host_per_layer_of_32": plan_host_ms / 32,   # one plan serves every layer of a step
         "pct_of_bf16_peak": {"measured": value / world / peaks["bf16_tflops"], "nominal": value / world / NOMINAL_BF16_TFLOPS,
                              "peak_source": peaks["source"]},
+        # the other bound of attention fwd+bwd: six passes over Hq-sized and six over Hkv-sized tensors
+        # (the short-many workload sits below the ridge point and is bounded by this one)
+        "attention_min_hbm": {"bytes": att_min_bytes, "gbs": att_min_bytes / att_ms / 1e6,
+                              "frac_of_hbm": {"measured": att_min_bytes / att_ms / 1e6 / peaks["hbm_gbs"],
+                                              "nominal": att_min_bytes / att_ms / 1e6 / NOMINAL_HBM_GBS}},
         "tokens_per_s": world * T / (step_ms * 1e-3),
         "attention_tokens_per_s": world * T / (att_ms * 1e-3),
         "kernels": {"psa_fwd_ms": fwd_ms, "psa_fwd_tflops": flops_fwd / fwd_ms / 1e9,
