@@ -10,6 +10,11 @@
 //                P = exp2(S*c - m*c) in fp32 and written back to TMEM as bf16 (over the thread's
 //                own S columns) for the second UMMA.  The two halves of a row exchange their
 //                maxima through shared memory.
+// A CTA takes two work items (query tile, query head), one after the other: items 2 b and 2 b + 1 of the list
+// (longest first; usually the same query tile and two heads of one kv head).  Barrier parities run on over both
+// items; the second item's Q and first K tile are requested as soon as the first item's last score product has
+// read them, i.e. they arrive while the first item's last softmax, P V and output store are still going on, and
+// the barrier initialisation, the TMEM allocation and the exit are paid once for two items.
 // Two CTAs share an SM (100 KB of shared memory and 256 TMEM columns each for head_dim 128), so
 // one CTA's softmax overlaps the other's UMMAs, and with eight softmax warps per CTA every SM
 // sub-partition has two warps feeding its exponential unit even when only one CTA is in that phase.
@@ -64,8 +69,16 @@ struct FwdParams {
   float* lse;
   int32_t* status;
   int32_t T, Hq, Hkv;
+  int32_t n_items;   // query tiles x query heads
   float scale_log2;  // softmax_scale * log2(e)
 };
+
+// What a role needs to know about one work item; both items of the CTA are kept in shared memory.
+struct FwdItem {
+  TileRec rec;
+  int32_t h, hk, n_it, pad;
+};
+static_assert(sizeof(FwdItem) == 48, "FwdItem is 12 int32");
 
 template <int D>
 struct FwdSmem {
@@ -73,19 +86,21 @@ struct FwdSmem {
   static constexpr int kTileBytes = kTile * D * 2;    // one Q / K / V tile
   static constexpr int kSubBytes = kTile * 128;       // one sub-tile: 128 rows x 128 bytes
   static constexpr int kQ = 0, kK = kTileBytes, kV = 2 * kTileBytes;
-  static constexpr int kBars = 3 * kTileBytes;        // 8 mbarriers
-  static constexpr int kTmemSlot = kBars + 64;
+  static constexpr int kBars = 3 * kTileBytes;        // 9 mbarriers
+  static constexpr int kTmemSlot = kBars + 72;
   static constexpr int kAbort = kTmemSlot + 4;
-  static constexpr int kEnt = kBars + 128;            // first kEntCap entries of the tile's list
+  static constexpr int kItems = kBars + 128;          // FwdItem [2]
+  static constexpr int kEnt = kItems + 128;           // first kEntCap entries of each item's list
   static constexpr int kEntCap = 128;
-  static constexpr int kXchg = kEnt + kEntCap * 4;    // float [2 parities][2 halves][128 rows]
+  static constexpr int kXchg = kEnt + 2 * kEntCap * 4;  // float [2 parities][2 halves][128 rows]
   static constexpr int kBytes = kXchg + 2 * 2 * kTile * 4;
   // Request enough that at most two CTAs fit on an SM: their TMEM allocations
   // (256 columns each) then always succeed without waiting.
   static constexpr int kRequest = (kBytes + 1024 > 100 * 1024) ? kBytes + 1024 : 100 * 1024;
 };
 
-enum { BAR_Q_FULL = 0, BAR_K_FULL, BAR_V_FULL, BAR_K_EMPTY, BAR_V_EMPTY, BAR_S_FULL, BAR_P_FULL, BAR_O_FULL };
+enum { BAR_Q_FULL = 0, BAR_K_FULL, BAR_V_FULL, BAR_K_EMPTY, BAR_V_EMPTY, BAR_S_FULL, BAR_P_FULL, BAR_O_FULL,
+       BAR_STAGE_FREE };   // the output staging (the V buffer) of the first item has been read by its TMA stores
 
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 2)
@@ -113,19 +128,45 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     g_psa_cta_trace_fwd[blockIdx.x * 4 + 2] = sm;
   }
 #endif
-  const int tile_idx = blockIdx.x / prm.Hq;
-  const int h = blockIdx.x % prm.Hq;
+  // The CTA's work items: 2 b and 2 b + 1 of the list (longest first, so the CTAs stay sorted by length and the
+  // short ones still fill the tail of the launch); the last CTA of an odd count has one item.
+  const int idx0 = 2 * int(blockIdx.x), idx1 = idx0 + 1;
+  const int n_items = idx1 < prm.n_items ? 2 : 1;
+  FwdItem* s_item = reinterpret_cast<FwdItem*>(gen_base + L::kItems);
+  int32_t* s_ent_all = reinterpret_cast<int32_t*>(gen_base + L::kEnt);
+  const WaitCtx wctx{abort_flag, prm.status};
+  // Every role reads the list entry of every iteration: the head of each item's list is kept in shared memory.
+  struct ItemView {
+    TileRec rec;
+    int h, hk, n_it;
+    const int32_t* ent_g;
+    const int32_t* s_ent;
+    __device__ __forceinline__ int ent(int it) const { return it < L::kEntCap ? s_ent[it] : ent_g[it]; }
+  };
+  auto view = [&](int item) {
+    const FwdItem im = s_item[item];
+    return ItemView{im.rec, im.h, im.hk, im.n_it, prm.entries + im.rec.list_off, s_ent_all + item * L::kEntCap};
+  };
+
+  if (threadIdx.x == 32 && n_items == 2) {   // the second item's record, while thread 0 requests the first tiles
+    const int h1 = idx1 % prm.Hq;
+    const TileRec r1 = prm.tiles[idx1 / prm.Hq];
+    s_item[1] = FwdItem{r1, h1, h1 / (prm.Hq / prm.Hkv), r1.list_cnt, 0};
+  }
+  if (threadIdx.x >= 128 && threadIdx.x < 128 + L::kEntCap && n_items == 2) {
+    const TileRec r1 = prm.tiles[idx1 / prm.Hq];
+    const int i = int(threadIdx.x) - 128;
+    if (i < r1.list_cnt) s_ent_all[L::kEntCap + i] = prm.entries[r1.list_off + i];
+  }
+  const int h = idx0 % prm.Hq;
   const int hk = h / (prm.Hq / prm.Hkv);
-  const TileRec rec = prm.tiles[tile_idx];
+  const TileRec rec = prm.tiles[idx0 / prm.Hq];
   const int32_t* ent_g = prm.entries + rec.list_off;
   const int n_it = rec.list_cnt;
-  int32_t* s_ent = reinterpret_cast<int32_t*>(gen_base + L::kEnt);
-  // Every role reads the list entry of every iteration: keep the head of the list in shared memory.
-  auto ent = [&](int it) { return it < L::kEntCap ? s_ent[it] : ent_g[it]; };
-  const WaitCtx wctx{abort_flag, prm.status};
-
   if (threadIdx.x == 0) {
     *abort_flag = 0;
+    s_item[0] = FwdItem{rec, h, hk, n_it, 0};
+    mbar_init(bar(BAR_STAGE_FREE), 1);
     mbar_init(bar(BAR_Q_FULL), 1);
     mbar_init(bar(BAR_K_FULL), 1);
     mbar_init(bar(BAR_V_FULL), 1);
@@ -151,7 +192,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
     tma_prefetch_desc(&tm_o);
   }
-  if (int(threadIdx.x) < n_it && int(threadIdx.x) < L::kEntCap) s_ent[threadIdx.x] = ent_g[threadIdx.x];
+  if (int(threadIdx.x) < n_it && int(threadIdx.x) < L::kEntCap) s_ent_all[threadIdx.x] = ent_g[threadIdx.x];
   if (warp == 0) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
   }
@@ -166,14 +207,27 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
    if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      for (int it = 1; it < n_it; ++it) {   // iteration 0 was requested before the CTA-wide barrier
-        const int krow = rec.ds + (ent(it) >> 2) * kTile;
-        mbar_wait(bar(BAR_K_EMPTY), (it - 1) & 1, wctx);
-        mbar_expect_tx(bar(BAR_K_FULL), L::kTileBytes);
-        for (int s = 0; s < L::kSub; ++s) tma_load_3d(sK + s * L::kSubBytes, &tm_k, s * 64, hk, krow, bar(BAR_K_FULL));
-        mbar_wait(bar(BAR_V_EMPTY), (it - 1) & 1, wctx);
-        mbar_expect_tx(bar(BAR_V_FULL), L::kTileBytes);
-        for (int s = 0; s < L::kSub; ++s) tma_load_3d(sV + s * L::kSubBytes, &tm_v, s * 64, hk, krow, bar(BAR_V_FULL));
+      int g = 0;   // iteration count over both items: the parity of every per-iteration barrier
+      for (int item = 0; item < n_items; ++item) {
+        const ItemView w = view(item);
+        for (int it = 0; it < w.n_it; ++it, ++g) {
+          if (g == 0) continue;   // requested before the CTA-wide barrier
+          const int krow = w.rec.ds + (w.ent(it) >> 2) * kTile;
+          mbar_wait(bar(BAR_K_EMPTY), (g - 1) & 1, wctx);
+          if (it == 0) {
+            // First tile of the second item.  The first item's last score product has completed, so
+            // its Q is no longer needed either.
+            mbar_expect_tx(bar(BAR_Q_FULL), L::kTileBytes);
+            for (int s = 0; s < L::kSub; ++s) tma_load_3d(sQ + s * L::kSubBytes, &tm_q, s * 64, w.h, w.rec.row0, bar(BAR_Q_FULL));
+          }
+          mbar_expect_tx(bar(BAR_K_FULL), L::kTileBytes);
+          for (int s = 0; s < L::kSub; ++s) tma_load_3d(sK + s * L::kSubBytes, &tm_k, s * 64, w.hk, krow, bar(BAR_K_FULL));
+          mbar_wait(bar(BAR_V_EMPTY), (g - 1) & 1, wctx);
+          // The first item's output leaves through the V buffer: its TMA stores must have read it.
+          if (it == 0) mbar_wait(bar(BAR_STAGE_FREE), 0, wctx);
+          mbar_expect_tx(bar(BAR_V_FULL), L::kTileBytes);
+          for (int s = 0; s < L::kSub; ++s) tma_load_3d(sV + s * L::kSubBytes, &tm_v, s * 64, w.hk, krow, bar(BAR_V_FULL));
+        }
       }
     }
     __syncwarp();
@@ -186,10 +240,13 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       constexpr uint32_t idesc_o = umma_idesc_bf16(kTile, D, false, true);       // P (TMEM), V MN-major
       // Low descriptor words (start address + LBO); the high word is a constant.
       const uint32_t q_k = smem_desc_lo(sQ, 16), k_k = smem_desc_lo(sK, 16), v_mn = smem_desc_lo(sV, L::kSubBytes);
-      mbar_wait(bar(BAR_Q_FULL), 0, wctx);
-      for (int it = 0; it < n_it; ++it) {
+      int g = 0;   // iteration count over both items
+      for (int item = 0; item < n_items; ++item) {
+      const ItemView w = view(item);
+      mbar_wait(bar(BAR_Q_FULL), item & 1, wctx);
+      for (int it = 0; it < w.n_it; ++it, ++g) {
         PSA_FWD_MARK(it, 0);
-        mbar_wait(bar(BAR_K_FULL), it & 1, wctx);
+        mbar_wait(bar(BAR_K_FULL), g & 1, wctx);
         PSA_FWD_MARK(it, 1);
         // The S columns are also where P_{it-1} lives.  UMMAs issued by one thread execute in
         // issue order, so this S = Q K^T cannot overwrite P before the previous P V has read it.
@@ -202,14 +259,14 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         umma_commit_w(bar(BAR_K_EMPTY), issuer);
         umma_commit_w(bar(BAR_S_FULL), issuer);
         PSA_FWD_MARK(it, 2);
-        mbar_wait(bar(BAR_V_FULL), it & 1, wctx);
+        mbar_wait(bar(BAR_V_FULL), g & 1, wctx);
         PSA_FWD_MARK(it, 3);
-        mbar_wait(bar(BAR_P_FULL), it & 1, wctx);
+        mbar_wait(bar(BAR_P_FULL), g & 1, wctx);
         PSA_FWD_MARK(it, 4);
         tc_fence_after();
         // P of key half hf lies in columns [64 hf, 64 hf + 32) of the S region (two bf16 per column);
         // PRECISE tiles carry a second bf16 term in columns [64 hf + 32, 64 hf + 64).
-        const int n_terms = (ent(it) & 2) ? 2 : 1;
+        const int n_terms = (w.ent(it) & 2) ? 2 : 1;
         for (int term = 0; term < n_terms; ++term) {
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk) {
@@ -222,6 +279,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         umma_commit_w(bar(BAR_O_FULL), issuer);
         PSA_FWD_MARK(it, 5);
       }
+      }
     }
     __syncwarp();
    }
@@ -233,11 +291,8 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const int r = quarter * 32 + lane;            // row within the tile
     const uint32_t lane_base = uint32_t(quarter * 32) << 16;
     const uint32_t col_s = kColS + 64u * hfz;     // this thread's 64 S columns; its P goes over them
-    const int q_local = rec.local0 + r;
-    const bool row_valid = q_local < rec.len;
     const float c = prm.scale_log2;
     float* xchg = reinterpret_cast<float*>(gen_base + L::kXchg);
-    float m_run = -INFINITY, l_run = 0.f;         // l_run: this thread's half of the row sum
     // Barrier of the two warps that share a row quarter (ids 1..4, immediate so that the kernel
     // is known to use five barriers, not all sixteen).
     auto pair_sync = [&]() {
@@ -249,11 +304,21 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
     };
 
-    for (int it = 0; it < n_it; ++it) {
-      const int e = ent(it);
+    int gbase = 0;       // iterations of the items before this one: barrier parities run on over both items
+    uint32_t xs = 0;     // uses of the exchange slots so far (they alternate with every use)
+    for (int item = 0; item < n_items; ++item) {
+    const ItemView w = view(item);
+    const TileRec& rec = w.rec;
+    const int h = w.h, n_it = w.n_it;
+    const int q_local = rec.local0 + r;
+    const bool row_valid = q_local < rec.len;
+    float m_run = -INFINITY, l_run = 0.f;         // l_run: this thread's half of the row sum
+    for (int it = 0; it < n_it; ++it, ++xs) {
+      const int g = gbase + it;
+      const int e = w.ent(it);
       const int k0 = (e >> 2) * kTile;
       const bool precise = (e & 2) != 0;
-      mbar_wait(bar(BAR_S_FULL), it & 1, wctx);
+      mbar_wait(bar(BAR_S_FULL), g & 1, wctx);
       tc_fence_after();
       if (threadIdx.x == 128) PSA_FWD_MARK(it, 6);
       if (threadIdx.x == 128 && it == 0) PSA_FWD_PHASE(2);
@@ -371,7 +436,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         float mxf = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         {
-          float* slot = xchg + (it & 1) * 2 * kTile;
+          float* slot = xchg + (xs & 1) * 2 * kTile;
           slot[hfz * kTile + r] = mxf;
           pair_sync();
           mxf = fmaxf(mxf, slot[(hfz ^ 1) * kTile + r]);
@@ -426,7 +491,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       // (slots alternate with the iteration parity, so a slot is rewritten only after the partner
       // has passed the next barrier, hence read it).
       {
-        float* slot = xchg + (it & 1) * 2 * kTile;
+        float* slot = xchg + (xs & 1) * 2 * kTile;
         slot[hfz * kTile + r] = mx;
         pair_sync();
         mx = fmaxf(mx, slot[(hfz ^ 1) * kTile + r]);
@@ -444,7 +509,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         l_run *= alpha;
       }
       if (it > 0 && __any_sync(0xffffffffu, grow)) {
-        mbar_wait(bar(BAR_O_FULL), (it - 1) & 1, wctx);
+        mbar_wait(bar(BAR_O_FULL), (g - 1) & 1, wctx);
         tc_fence_after();
         // Each thread rescales its half of the accumulator's columns.
 #pragma unroll
@@ -535,20 +600,21 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (threadIdx.x == 128) PSA_FWD_PHASE(4);
     // ---- epilogue: O / l -> bf16, lse.  The two halves of the row sum meet in shared memory.
     {
-      float* slot = xchg + (n_it & 1) * 2 * kTile;
+      float* slot = xchg + (xs & 1) * 2 * kTile;
+      ++xs;
       slot[hfz * kTile + r] = l_run;
       pair_sync();
       l_run += slot[(hfz ^ 1) * kTile + r];
     }
     if (n_it > 0) {
-      mbar_wait(bar(BAR_O_FULL), (n_it - 1) & 1, wctx);
+      mbar_wait(bar(BAR_O_FULL), (gbase + n_it - 1) & 1, wctx);
       tc_fence_after();
     }
     if (threadIdx.x == 128) PSA_FWD_PHASE(5);
     const float inv_l = 1.f / l_run;
     const int64_t row = int64_t(rec.row0) + r;
     __nv_bfloat16* orow = prm.o + (row * prm.Hq + h) * D + hfz * (D / 2);
-    // A full tile leaves through shared memory (the Q buffer is free now) in the 128-byte-swizzled
+    // A full tile leaves through shared memory (the V buffer is free now) in the 128-byte-swizzled
     // layout of the tensor map and one TMA store per 64-column sub-tile writes it out coalesced.
     // (A ragged last tile must not touch the rows of the next sample, which the box would cover:
     // it takes the per-thread stores.)
@@ -559,7 +625,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       tmem_ld32_wait(tmem + lane_base + kColO + hfz * (D / 2) + ch * 32, v);
       if (full_tile) {
         const int col0 = hfz * (D / 2) + ch * 32;
-        const uint32_t row_addr = sQ + (col0 >> 6) * L::kSubBytes + r * 128;
+        const uint32_t row_addr = sV + (col0 >> 6) * L::kSubBytes + r * 128;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint32_t chunk = uint32_t(((col0 & 63) >> 3) + i) ^ uint32_t(r & 7);
@@ -590,11 +656,15 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       fence_proxy_async_smem();
       asm volatile("bar.sync 5, 256;" ::: "memory");   // the eight softmax warps
       if (threadIdx.x == 128) {
-        for (int s = 0; s < L::kSub; ++s) tma_store_3d(&tm_o, sQ + s * L::kSubBytes, s * 64, h, rec.row0);
+        for (int s = 0; s < L::kSub; ++s) tma_store_3d(&tm_o, sV + s * L::kSubBytes, s * 64, h, rec.row0);
         tma_commit_group();
         tma_wait_group_read<0>();   // shared memory must outlive the stores' reads
       }
     }
+    // The V buffer may be refilled (by the next item's first V tile) once the stores have read it.
+    if (threadIdx.x == 128 && item == 0) mbar_arrive(bar(BAR_STAGE_FREE));
+    gbase += n_it;
+    }   // items
     if (threadIdx.x == 128) PSA_FWD_PHASE(6);
   }
 
@@ -633,8 +703,9 @@ psa_status_t launch_fwd_t(const psa_plan_t* plan, const void* q, const void* k, 
   prm.T = plan->T;
   prm.Hq = plan->Hq;
   prm.Hkv = plan->Hkv;
+  prm.n_items = int32_t(plan->q_tiles.size()) * plan->Hq;
   prm.scale_log2 = plan->scale * 1.4426950408889634f;
-  const unsigned grid = unsigned(plan->q_tiles.size()) * unsigned(plan->Hq);
+  const unsigned grid = unsigned(prm.n_items + 1) / 2u;   // two work items per CTA
   {
     ProfileScope prof(0, stream);
     psa_fwd_kernel<D><<<grid, kFwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, tm_o, prm);
