@@ -368,6 +368,50 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       // that the running maximum still holds (it nearly always does, see the 2^8 rule below).
       // If it does not, nothing has been written yet and the two-pass path below redoes the tile.
       bool fast_done = false;
+      if (it == 0 && !precise && cls == 0u) {
+        // First tile of a list, nothing masked: there is no accumulator to rescale yet, so the
+        // scores can stay in registers across the exchange of the maxima (one load instead of three).
+        uint32_t v[64];
+        tmem_ld64_wait(tmem + lane_base + col_s, v);
+        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int i = 0; i < 64; i += 8) {
+          m4[0] = max3(m4[0], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
+          m4[1] = max3(m4[1], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+          m4[2] = max3(m4[2], __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+          m4[3] = max3(m4[3], __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+        }
+        float mxf = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        {
+          float* slot = xchg + (xs & 1) * 2 * kTile;
+          slot[hfz * kTile + r] = mxf;
+          pair_sync();
+          mxf = fmaxf(mxf, slot[(hfz ^ 1) * kTile + r]);
+        }
+        m_run = mxf;
+        const float mc0 = (m_run == -INFINITY) ? 0.f : m_run * c;
+        const uint64_t c2 = pack_f32x2(c, c), mc2 = pack_f32x2(-mc0, -mc0);
+        uint64_t sum2[2] = {0ull, 0ull};
+        uint32_t pk[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          float t0, t1;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])), c2, mc2), t0, t1);
+          const float p0 = ex2_approx(t0), p1 = ex2_approx(t1);
+          sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(p0, p1));
+          pk[i] = pack_bf16x2(p0, p1);
+        }
+        tmem_st32(tmem + lane_base + col_s, pk);
+        float a0, a1, b0, b1;
+        unpack_f32x2(sum2[0], a0, a1);
+        unpack_f32x2(sum2[1], b0, b1);
+        l_run = (a0 + a1) + (b0 + b1);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_P_FULL));
+        if (threadIdx.x == 128) PSA_FWD_MARK(it, 9);
+        continue;
+      }
       if (it > 0 && !precise) {
         uint32_t pk[32];
         float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
