@@ -363,10 +363,10 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
       };
       // Fast path (every tile but the first of a list and the PRECISE ones): one pass.  The
-      // exponentials are taken against the running maximum while the tile's own maximum is
-      // found on the side; P stays in registers until the two threads of the row have agreed
-      // that the running maximum still holds (it nearly always does, see the 2^8 rule below).
-      // If it does not, nothing has been written yet and the two-pass path below redoes the tile.
+      // exponentials are taken against the running maximum; P stays in registers until the two
+      // threads of the row have agreed that the running maximum still holds (it nearly always
+      // does, see the 2^8 rule below).  If it does not, nothing has been written yet and the
+      // two-pass path below redoes the tile.
       bool fast_done = false;
       if (it == 0 && !precise && cls == 0u) {
         // First tile of a list, nothing masked: there is no accumulator to rescale yet, so the
@@ -414,7 +414,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       if (it > 0 && !precise) {
         uint32_t pk[32];
-        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         uint64_t sum2[2] = {0ull, 0ull};
         const float mc0 = (m_run == -INFINITY) ? 0.f : m_run * c;
         const uint64_t c2 = pack_f32x2(c, c), mc2 = pack_f32x2(-mc0, -mc0);
@@ -423,13 +422,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           // wait exposes the TMEM latency, which the two warps per sub-partition do not hide.
           uint32_t v[64];
           tmem_ld64_wait(tmem + lane_base + col_s, v);
-#pragma unroll
-          for (int i = 0; i < 64; i += 8) {
-            m4[0] = max3(m4[0], __uint_as_float(v[i]), __uint_as_float(v[i + 1]));
-            m4[1] = max3(m4[1], __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-            m4[2] = max3(m4[2], __uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
-            m4[3] = max3(m4[3], __uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
-          }
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             float t0, t1;
@@ -463,13 +455,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             for (int i = 0; i < 16; ++i) x[i] = __uint_as_float(v[i]);
           }
 #pragma unroll
-          for (int i = 0; i < 16; i += 8) {
-            m4[0] = max3(m4[0], x[i], x[i + 1]);
-            m4[1] = max3(m4[1], x[i + 2], x[i + 3]);
-            m4[2] = max3(m4[2], x[i + 4], x[i + 5]);
-            m4[3] = max3(m4[3], x[i + 6], x[i + 7]);
-          }
-#pragma unroll
           for (int i = 0; i < 8; ++i) {
             float t0, t1;
             unpack_f32x2(fma_f32x2(pack_f32x2(x[2 * i], x[2 * i + 1]), c2, mc2), t0, t1);
@@ -478,21 +463,25 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             pk[8 * ch + i] = pack_bf16x2(p0, p1);
           }
         }
-        float mxf = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        // The running maximum still holds if no probability of the tile exceeds 2^8 against it.  The
+        // row sum, which is needed anyway, bounds them all: above 256 (or not a number, or a first
+        // contribution to a row whose running maximum is still -inf) the tile goes to the two-pass path.
+        float a0, a1, b0, b1;
+        unpack_f32x2(sum2[0], a0, a1);
+        unpack_f32x2(sum2[1], b0, b1);
+        const float sumf = (a0 + a1) + (b0 + b1);
+        bool redo = !(sumf <= 256.f) || (m_run == -INFINITY && sumf > 0.f);
         {
+          // both threads of a row must take the same path
           float* slot = xchg + (xs & 1) * 2 * kTile;
-          slot[hfz * kTile + r] = mxf;
+          slot[hfz * kTile + r] = redo ? 1.f : 0.f;
           pair_sync();
-          mxf = fmaxf(mxf, slot[(hfz ^ 1) * kTile + r]);
+          redo = redo || slot[(hfz ^ 1) * kTile + r] != 0.f;
         }
-        const bool grow_f = (fmaxf(m_run, mxf) - m_run) * c > 8.0f;
-        if (!__any_sync(0xffffffffu, grow_f)) {
+        if (!__any_sync(0xffffffffu, redo)) {
           // the 16 values of chunk ch go to columns [8 ch, 8 ch + 8) of the thread's own 64
           tmem_st32(tmem + lane_base + col_s, pk);
-          float a0, a1, b0, b1;
-          unpack_f32x2(sum2[0], a0, a1);
-          unpack_f32x2(sum2[1], b0, b1);
-          l_run += (a0 + a1) + (b0 + b1);
+          l_run += sumf;
           tc_wait_st();
           tc_fence_before();
           mbar_arrive(bar(BAR_P_FULL));
