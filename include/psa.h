@@ -45,8 +45,8 @@ typedef enum {
   PSA_ERR_UNSUPPORTED = 3,          /* head_dim not in {64,128}, Hq % Hkv != 0, size over a stated maximum */
   PSA_ERR_ALIGNMENT = 4,            /* a device pointer is not 16-byte aligned */
   PSA_ERR_CUDA = 5,                 /* a CUDA runtime / driver call failed (no device, launch error, ...) */
-  PSA_ERR_DEVICE_STATUS = 6,        /* reserved: a kernel reported bad data through a status word */
-  PSA_ERR_TIMEOUT = 7               /* reserved: a bounded device-side wait expired */
+  PSA_ERR_DEVICE_STATUS = 6,        /* psa_check_device_status: a kernel reported bad data (labels) */
+  PSA_ERR_TIMEOUT = 7               /* psa_check_device_status: a bounded device-side wait expired  */
 } psa_status_t;
 
 /* Bits of the word a kernel ORs into `device_status` (device int32, may be NULL). */
@@ -58,6 +58,26 @@ typedef enum {
 #define PSA_PLAN_HOST_ONLY 1 /* build the tile map on the host only; no CUDA call is made */
 
 const char* psa_status_string(psa_status_t s);
+
+/*
+ * psa_check_device_status -- turns a device status word (copied back to the host by the
+ * caller, after the stream has been synchronised) into a status code: 0 -> PSA_OK;
+ * PSA_DEVSTAT_WAIT_EXPIRED set -> PSA_ERR_TIMEOUT (the outputs of that call are invalid);
+ * otherwise a label bit set -> PSA_ERR_DEVICE_STATUS.  Host only; no paper counterpart.
+ */
+psa_status_t psa_check_device_status(int32_t device_status_word);
+
+/*
+ * psa_selftest_wait_expiry -- failure-detection self test; the paper has no counterpart.
+ * Launches one small CTA that waits, with the same bounded wait the attention kernels use, on
+ * a barrier that nothing will ever complete.  After `limit_clocks` SM clocks (clamped to
+ * [1e3, 4e9]) the wait gives up, ORs PSA_DEVSTAT_WAIT_EXPIRED into *device_status and the
+ * kernel returns normally: the context stays usable.  Nothing faults, traps or spins without
+ * a limit.  `spins_out` (device int64, may be NULL) receives the clocks the wait lasted.
+ * Errors: INVALID_ARG (device_status NULL), CUDA.
+ */
+psa_status_t psa_selftest_wait_expiry(int32_t* device_status, int64_t limit_clocks, int64_t* spins_out,
+                                      void* stream);
 
 /*
  * psa_plan -- build the block-sparsity tile map of the Algorithm 3 mask once per
@@ -144,7 +164,8 @@ psa_status_t psa_plan_export(const psa_plan_t* plan, int32_t direction,
  *   o        device bf16 [T, Hq, d] (out)  lse    device fp32 [Hq, T] (out)
  *   device_status  device int32 or NULL; bits are ORed in, never cleared.
  * Rows >= T are neither read nor written.  T = 0 is a no-op.
- * Errors: INVALID_ARG, ALIGNMENT, CUDA.
+ * Errors: INVALID_ARG (also: the plan was uploaded on another device than the current one),
+ * ALIGNMENT, CUDA.
  */
 psa_status_t psa_fwd(const psa_plan_t* plan, const void* q, const void* k, const void* v,
                      void* o, float* lse, int32_t* device_status, void* stream);
@@ -166,6 +187,22 @@ psa_status_t psa_bwd(const psa_plan_t* plan, const void* d_o, const void* q, con
                      const void* v, const void* o, const float* lse,
                      void* dq, void* dk, void* dv, void* workspace,
                      int32_t* device_status, void* stream);
+
+/*
+ * psa_bwd_f32 -- psa_bwd with fp32 gradient outputs (same computation, same kernels; the only
+ * difference is that the fp32 accumulators are written out as they are instead of being rounded
+ * to bf16).  For callers that accumulate gradients in fp32, and for checking the gradients
+ * against a reference without the bf16 output rounding in the way.
+ *   dq          device fp32 [T, Hq, d] (out): serves as the accumulator itself
+ *   dk, dv      device fp32 [T, Hkv, d] (out)
+ *   workspace   as for psa_bwd (same size; only its delta part is used)
+ *   everything else as for psa_bwd.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA.
+ */
+psa_status_t psa_bwd_f32(const psa_plan_t* plan, const void* d_o, const void* q, const void* k,
+                         const void* v, const void* o, const float* lse,
+                         float* dq, float* dk, float* dv, void* workspace,
+                         int32_t* device_status, void* stream);
 
 /*
  * psa_bwd_static_scratch -- psa_bwd without the workspace argument.  The paper has no
@@ -299,6 +336,60 @@ psa_status_t psa_rope(const void* x, void* y, const int32_t* position_ids, int64
  */
 psa_status_t psa_pack_ffd(const int32_t* unit_len, int32_t n_units, int32_t capacity,
                           int32_t* bin_of_unit, int32_t* n_bins);
+
+/*
+ * psa_pack_ffd_emit -- psa_pack_ffd followed by the lay-out of every pack in the form psa_plan
+ * takes (Section 3.2: the prompt and its two responses are packed as one unit; Section 4.3.2).
+ * Host only, no CUDA call.
+ *   prefix_len, chosen_len, rejected_len   host int32 [n_units]: P, C, R of each sample
+ *   capacity     the packing length
+ *   paired       0: shared layout, one sample (P, C, R) of P + C + R tokens per unit;
+ *                1: the unshared baseline layout, two samples (P, C, 0) and (P, R, 0) per unit,
+ *                   kept next to each other in one pack (unit length 2P + C + R)
+ *   bin_of_unit  host int32 [n_units] (out): the pack of each unit, as psa_pack_ffd
+ *   n_packs      host int32 (out)
+ *   pack_sample_offset   host int32 [n_units + 1] (out; n_packs + 1 entries written): the samples
+ *                of pack b are entries [off[b], off[b+1]) of the four arrays below
+ *   sample_unit  host int32 [m] (out), m = n_units (shared) or 2 n_units (paired): the unit a
+ *                sample came from.  Within a pack the units stand in the order the packer placed
+ *                them (longest first, ties by index).
+ *   out_prefix_len, out_chosen_len, out_rejected_len   host int32 [m] (out)
+ *   out_cu_seqlens   host int32 [m + n_units] (out): the packs' cu_seqlens arrays one after the
+ *                other; pack b's array starts at index off[b] + b and has off[b+1] - off[b] + 1
+ *                entries, the first of them 0.
+ * Pack b is planned with
+ *   psa_plan(out_cu_seqlens + off[b] + b, out_prefix_len + off[b], out_chosen_len + off[b],
+ *            out_rejected_len + off[b], off[b+1] - off[b], ...).
+ * Errors: INVALID_ARG, UNSUPPORTED (a unit is longer than the capacity; nothing is written).
+ */
+psa_status_t psa_pack_ffd_emit(const int32_t* prefix_len, const int32_t* chosen_len,
+                               const int32_t* rejected_len, int32_t n_units, int32_t capacity,
+                               int32_t paired, int32_t* bin_of_unit, int32_t* n_packs,
+                               int32_t* pack_sample_offset, int32_t* sample_unit,
+                               int32_t* out_prefix_len, int32_t* out_chosen_len,
+                               int32_t* out_rejected_len, int32_t* out_cu_seqlens);
+
+/*
+ * psa_logp_labels -- which logits row scores which token on the shared layout, for dpo_logp
+ * (Section 2.1: the log-probs are those of the paired format; Section 3.2: responses are
+ * recovered from their boundaries).  The paper gives no formula; the reading is next-token
+ * scoring inside each response's own context: row t scores token t + 1 of the same response;
+ * the last prompt row scores BOTH the first chosen and the first rejected token (the second of
+ * the two labels goes to the fork list); the last chosen and the last rejected row score nothing;
+ * with an empty prompt the first token of a response has no scoring row.  Host only.
+ *   token_ids    host int32 [T]: the packed row's tokens
+ *   cu_seqlens, prefix_len, chosen_len, rejected_len, n_samples   as for psa_plan
+ *   targets, segment_ids   host int32 [T] (out): label and response id (2s chosen, 2s+1
+ *                rejected, -1 none) of each row, as dpo_logp takes them
+ *   fork_rows, fork_targets, fork_segments   host int32 [n_samples] (out; n_forks entries written)
+ *   n_forks      host int32 (out)
+ * Errors: INVALID_ARG, INCONSISTENT_LENGTHS.
+ */
+psa_status_t psa_logp_labels(const int32_t* token_ids, const int32_t* cu_seqlens,
+                             const int32_t* prefix_len, const int32_t* chosen_len,
+                             const int32_t* rejected_len, int32_t n_samples, int32_t* targets,
+                             int32_t* segment_ids, int32_t* fork_rows, int32_t* fork_targets,
+                             int32_t* fork_segments, int32_t* n_forks);
 
 /*
  * dpo_loss -- the DPO loss of Eq. 1 (Section 2.1) from the four summed log-probs per sample.

@@ -11,10 +11,10 @@ only library primitive used as a step.
 
 Paper passages each function follows:
 
-* ``token_metadata`` / ``prefix_sharing_mask_packed``: Algorithm 3 ("Prefix
+* ``token_roles`` / ``prefix_sharing_mask_packed``: Algorithm 3 ("Prefix
   Sharing Mask with Packing"): causal AND same-document AND NOT(rejected query
-  looking at a chosen key), with dense per-token arrays I_chosen, I_rejected
-  and document ids D (Section 3.2).
+  looking at a chosen key), from dense per-token arrays (sample id and
+  prompt / chosen / rejected role of every token, Section 3.2).
 * ``prefix_sharing_mask_single``: Algorithm 1 ("Prefix Sharing Mask").
 * ``paired_packing_mask``: Algorithm 2 ("Attention Mask for Packing w/o Prefix
   Sharing"): causal AND same per-token response id.
@@ -47,68 +47,62 @@ import numpy as np
 # Masks
 # --------------------------------------------------------------------------
 
-def token_metadata(cu_seqlens, prefix_len, chosen_len, rejected_len):
-    """Dense per-token arrays of Algorithm 3 for one packed row (B = 1, L = T).
+PROMPT, CHOSEN, REJECTED = 0, 1, 2
 
-    Returns (D, I_chosen, I_rejected), each int64 [T]: the document id of the
-    token's sample and the absolute start index, in the packed row, of that
-    sample's chosen and rejected completions.
-    """
+
+def token_roles(cu_seqlens, prefix_len, chosen_len, rejected_len):
+    """Per-token description of one packed row: which sample a token belongs to and whether it
+    is a prompt, chosen or rejected token.  (Algorithm 3 carries the same information as a
+    document id and two start indices per token, Section 3.2.)  Returns (sample_of, role),
+    each int64 [T]."""
     cu = np.asarray(cu_seqlens, dtype=np.int64)
     n = len(cu) - 1
     T = int(cu[n])
-    D = np.empty(T, dtype=np.int64)
-    Ic = np.empty(T, dtype=np.int64)
-    Ir = np.empty(T, dtype=np.int64)
+    sample_of = np.empty(T, dtype=np.int64)
+    role = np.empty(T, dtype=np.int64)
     for s in range(n):
         P, C, R = int(prefix_len[s]), int(chosen_len[s]), int(rejected_len[s])
         lo, hi = int(cu[s]), int(cu[s + 1])
         if hi - lo != P + C + R:
             raise ValueError("sample %d: cu_seqlens span %d != P+C+R = %d" % (s, hi - lo, P + C + R))
-        D[lo:hi] = s
-        Ic[lo:hi] = lo + P
-        Ir[lo:hi] = lo + P + C
-    return D, Ic, Ir
+        sample_of[lo:hi] = s
+        role[lo:lo + P] = PROMPT
+        role[lo + P:lo + P + C] = CHOSEN
+        role[lo + P + C:hi] = REJECTED
+    return sample_of, role
 
 
-def prefix_sharing_mask_packed(D, I_chosen, I_rejected):
-    """Algorithm 3, evaluated for every (q, kv) pair of the packed row.
-
-    mask[q, kv] = (kv <= q) and (D[q] == D[kv])
-                  and not ((I_rejected[q] <= q) and (I_chosen[q] <= kv < I_rejected[q]))
-    """
-    T = len(D)
-    q = np.arange(T, dtype=np.int64)[:, None]
-    kv = np.arange(T, dtype=np.int64)[None, :]
-    causal_mask = kv <= q
-    document_mask = D[:, None] == D[None, :]
-    chosen_ind = I_chosen[:, None]
-    rejected_ind = I_rejected[:, None]
-    dpo_mask = ~((rejected_ind <= q) & (chosen_ind <= kv) & (kv < rejected_ind))
-    return causal_mask & document_mask & dpo_mask
+def prefix_sharing_mask_packed(sample_of, role):
+    """The mask of Algorithm 3 over every (query, key) pair of the packed row: a query sees a
+    key iff the key is not after it, both belong to the same sample, and it is not the case
+    that the query is a rejected token while the key is a chosen token."""
+    T = len(role)
+    pos = np.arange(T, dtype=np.int64)
+    not_later = pos[None, :] <= pos[:, None]                       # [query, key]
+    same_sample = sample_of[:, None] == sample_of[None, :]
+    rejected_sees_chosen = (role[:, None] == REJECTED) & (role[None, :] == CHOSEN)
+    return not_later & same_sample & ~rejected_sees_chosen
 
 
-def prefix_sharing_mask_single(L, chosen_ind, rejected_ind):
-    """Algorithm 1 for one unpacked sample of length L (scalar start indices)."""
-    q = np.arange(L, dtype=np.int64)[:, None]
-    kv = np.arange(L, dtype=np.int64)[None, :]
-    causal_mask = kv <= q
-    dpo_mask = ~((rejected_ind <= q) & (chosen_ind <= kv) & (kv < rejected_ind))
-    return causal_mask & dpo_mask
+def prefix_sharing_mask_single(L, chosen_start, rejected_start):
+    """Algorithm 1: one unpacked sample of length L whose chosen response starts at
+    chosen_start and whose rejected response starts at rejected_start."""
+    pos = np.arange(L, dtype=np.int64)
+    role = np.where(pos < chosen_start, PROMPT, np.where(pos < rejected_start, CHOSEN, REJECTED))
+    return prefix_sharing_mask_packed(np.zeros(L, dtype=np.int64), role)
 
 
 def paired_packing_mask(response_ids):
-    """Algorithm 2: causal AND equal per-token response ids (paired layout)."""
-    Rid = np.asarray(response_ids, dtype=np.int64)
-    T = len(Rid)
-    q = np.arange(T, dtype=np.int64)[:, None]
-    kv = np.arange(T, dtype=np.int64)[None, :]
-    return (kv <= q) & (Rid[:, None] == Rid[None, :])
+    """Algorithm 2 (the paired baseline layout, packed): a query sees the keys of its own
+    sequence that are not after it; `response_ids` names the sequence of every token."""
+    ids = np.asarray(response_ids, dtype=np.int64)
+    pos = np.arange(len(ids), dtype=np.int64)
+    return (pos[None, :] <= pos[:, None]) & (ids[:, None] == ids[None, :])
 
 
 def packed_mask(cu_seqlens, prefix_len, chosen_len, rejected_len):
     """Convenience: Algorithm 3's mask straight from the per-sample lengths."""
-    return prefix_sharing_mask_packed(*token_metadata(cu_seqlens, prefix_len, chosen_len, rejected_len))
+    return prefix_sharing_mask_packed(*token_roles(cu_seqlens, prefix_len, chosen_len, rejected_len))
 
 
 def useful_pairs(prefix_len, chosen_len, rejected_len):

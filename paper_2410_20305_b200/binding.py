@@ -25,7 +25,8 @@ EXPORTED_SYMBOLS = (
     "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
     "psa_plan_counts", "psa_plan_export", "psa_fwd", "psa_bwd", "dpo_logp", "psa_profile_events",
     "psa_bwd_static_scratch", "dpo_loss", "dpo_logp_bwd", "psa_pack_ffd", "psa_position_ids", "psa_rope",
-    "psa_step_host_arena_bytes", "psa_step_host", "simpo_loss", "orpo_loss",
+    "psa_step_host_arena_bytes", "psa_step_host", "simpo_loss", "orpo_loss", "psa_bwd_f32",
+    "psa_check_device_status", "psa_selftest_wait_expiry", "psa_logp_labels", "psa_pack_ffd_emit",
 )
 
 
@@ -63,6 +64,11 @@ def load_library():
     lib.psa_fwd.argtypes = [vp] * 8
     lib.psa_bwd.argtypes = [vp] * 13
     lib.psa_bwd_static_scratch.argtypes = [vp] * 12
+    lib.psa_bwd_f32.argtypes = [vp] * 13
+    lib.psa_check_device_status.argtypes = [i32]
+    lib.psa_selftest_wait_expiry.argtypes = [vp, i64, vp, vp]
+    lib.psa_logp_labels.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, C.POINTER(i32)]
+    lib.psa_pack_ffd_emit.argtypes = [vp, vp, vp, i32, i32, i32, vp, C.POINTER(i32), vp, vp, vp, vp, vp, vp]
     lib.psa_profile_events.argtypes = [i32, vp, vp]
     lib.dpo_loss.argtypes = [vp, vp, i32, f32, vp, vp, vp]
     lib.simpo_loss.argtypes = [vp, vp, i32, f32, f32, vp, vp, vp, vp]
@@ -101,6 +107,35 @@ def _stream(stream):
 
 def _ptr(t):
     return C.c_void_p(0) if t is None else C.c_void_p(t.data_ptr())
+
+
+def _want(t, name, shape, dtype, cuda=True):
+    """Raises ValueError unless tensor `t` has exactly this shape and dtype, is contiguous and
+    lives where the call needs it.  The kernels size their tensor maps and grids from the plan
+    alone, so a tensor of another pack, or a buffer that is too small, would be read or written
+    past its end: it has to be refused here."""
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError("%s: shape %s, the plan needs %s" % (name, tuple(t.shape), tuple(shape)))
+    if t.dtype != dtype:
+        raise ValueError("%s: dtype %s, expected %s" % (name, t.dtype, dtype))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    if bool(t.is_cuda) != bool(cuda):
+        raise ValueError("%s must be a %s tensor" % (name, "CUDA" if cuda else "host"))
+
+
+def _want_attention(plan, bf16, f32=(), lse=None, cuda=True, grads_f32=False):
+    """Shape / dtype checks of the attention tensors against the plan: names in `bf16` are
+    (name, tensor, "q" or "kv") triples."""
+    import torch
+    T, d = plan.total_tokens, plan.head_dim
+    heads = {"q": plan.n_q_heads, "kv": plan.n_kv_heads}
+    for name, t, kind in bf16:
+        _want(t, name, (T, heads[kind], d), torch.bfloat16, cuda)
+    for name, t, kind in f32:
+        _want(t, name, (T, heads[kind], d), torch.float32, cuda)
+    if lse is not None:
+        _want(lse, "lse", (plan.n_q_heads, T), torch.float32, cuda)
 
 
 class Plan:
@@ -162,13 +197,12 @@ def psa_fwd(plan: Plan, q, k, v, o=None, lse=None, status=None, stream=None):
     """q [T,Hq,d], k, v [T,Hkv,d] bf16 CUDA tensors -> (o [T,Hq,d] bf16, lse [Hq,T] fp32)."""
     import torch
     T = plan.total_tokens
-    assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous() and tuple(q.shape) == (T, plan.n_q_heads, plan.head_dim)
-    for t in (k, v):
-        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and tuple(t.shape) == (T, plan.n_kv_heads, plan.head_dim)
+    _want_attention(plan, [("q", q, "q"), ("k", k, "kv"), ("v", v, "kv")])
     if o is None:
         o = torch.empty_like(q)
     if lse is None:
         lse = torch.empty((plan.n_q_heads, T), dtype=torch.float32, device=q.device)
+    _want_attention(plan, [("o", o, "q")], lse=lse)
     _check("psa_fwd", load_library().psa_fwd(plan._h, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(status),
                                              _stream(stream)))
     return o, lse
@@ -177,22 +211,56 @@ def psa_fwd(plan: Plan, q, k, v, o=None, lse=None, status=None, stream=None):
 def psa_bwd(plan: Plan, d_o, q, k, v, o, lse, dq=None, dk=None, dv=None, workspace=None, status=None, stream=None):
     """Returns (dq [T,Hq,d], dk, dv [T,Hkv,d]) bf16."""
     import torch
-    for t in (d_o, q, k, v, o):
-        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
-    assert lse.dtype == torch.float32 and lse.is_contiguous()
+    _want_attention(plan, [("d_o", d_o, "q"), ("q", q, "q"), ("k", k, "kv"), ("v", v, "kv"), ("o", o, "q")], lse=lse)
     if dq is None:
         dq = torch.empty_like(q)
     if dk is None:
         dk = torch.empty_like(k)
     if dv is None:
         dv = torch.empty_like(v)
+    _want_attention(plan, [("dq", dq, "q"), ("dk", dk, "kv"), ("dv", dv, "kv")])
     if workspace is None:
         workspace = torch.empty(max(plan.bwd_workspace_bytes, 256), dtype=torch.uint8, device=q.device)
-    assert workspace.numel() * workspace.element_size() >= plan.bwd_workspace_bytes
+    if not workspace.is_cuda or workspace.numel() * workspace.element_size() < plan.bwd_workspace_bytes:
+        raise ValueError("workspace: a CUDA buffer of at least %d bytes is needed" % plan.bwd_workspace_bytes)
     _check("psa_bwd", load_library().psa_bwd(plan._h, _ptr(d_o), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
                                              _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace), _ptr(status),
                                              _stream(stream)))
     return dq, dk, dv
+
+
+def psa_bwd_f32(plan: Plan, d_o, q, k, v, o, lse, dq=None, dk=None, dv=None, workspace=None, status=None, stream=None):
+    """psa_bwd with fp32 gradient outputs: returns (dq [T,Hq,d], dk, dv [T,Hkv,d]) fp32, the
+    kernels' fp32 accumulators written out without the final rounding to bf16."""
+    import torch
+    _want_attention(plan, [("d_o", d_o, "q"), ("q", q, "q"), ("k", k, "kv"), ("v", v, "kv"), ("o", o, "q")], lse=lse)
+    f32 = lambda t: torch.empty(t.shape, dtype=torch.float32, device=t.device)
+    dq = f32(q) if dq is None else dq
+    dk = f32(k) if dk is None else dk
+    dv = f32(v) if dv is None else dv
+    _want_attention(plan, [], f32=[("dq", dq, "q"), ("dk", dk, "kv"), ("dv", dv, "kv")])
+    if workspace is None:
+        workspace = torch.empty(max(plan.bwd_workspace_bytes, 256), dtype=torch.uint8, device=q.device)
+    if not workspace.is_cuda or workspace.numel() * workspace.element_size() < plan.bwd_workspace_bytes:
+        raise ValueError("workspace: a CUDA buffer of at least %d bytes is needed" % plan.bwd_workspace_bytes)
+    _check("psa_bwd_f32", load_library().psa_bwd_f32(plan._h, _ptr(d_o), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
+                                                     _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace), _ptr(status),
+                                                     _stream(stream)))
+    return dq, dk, dv
+
+
+def psa_check_device_status(word: int) -> int:
+    """Status code for a device status word read back by the caller: 0 ok, 7 a bounded wait
+    expired (outputs invalid), 6 bad labels."""
+    return int(load_library().psa_check_device_status(int(word)))
+
+
+def psa_selftest_wait_expiry(status, limit_clocks, waited=None, stream=None):
+    """Runs the library's bounded wait on a barrier that nothing completes; after `limit_clocks`
+    SM clocks the wait gives up and ORs PSA_DEVSTAT_WAIT_EXPIRED into `status` (int32 CUDA [1]).
+    `waited` (int64 CUDA [1], optional) receives the clocks the wait lasted."""
+    _check("psa_selftest_wait_expiry",
+           load_library().psa_selftest_wait_expiry(_ptr(status), int(limit_clocks), _ptr(waited), _stream(stream)))
 
 
 def dpo_logp(logits, targets, segment_ids, n_segments, fork_rows=None, fork_targets=None, fork_segments=None,
@@ -238,10 +306,8 @@ def psa_bwd_static_scratch(plan: Plan, d_o, q, k, v, o, lse, dq, dk, dv, status=
     array inside the library.  Nothing is allocated here either: the three gradient tensors
     must be passed in.  Plans whose scratch need exceeds PSA_STATIC_SCRATCH_BYTES raise
     PsaError (status 3).  Calls that overlap on the GPU share the array and must be serialised."""
-    import torch
-    for t in (d_o, q, k, v, o, dq, dk, dv):
-        assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
-    assert lse.dtype == torch.float32 and lse.is_contiguous()
+    _want_attention(plan, [("d_o", d_o, "q"), ("q", q, "q"), ("k", k, "kv"), ("v", v, "kv"), ("o", o, "q"),
+                           ("dq", dq, "q"), ("dk", dk, "kv"), ("dv", dv, "kv")], lse=lse)
     _check("psa_bwd_static_scratch",
            load_library().psa_bwd_static_scratch(plan._h, _ptr(d_o), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse),
                                                  _ptr(dq), _ptr(dk), _ptr(dv), _ptr(status), _stream(stream)))
@@ -259,10 +325,11 @@ def psa_step_host(plan: Plan, h_q, h_k, h_v, h_do, h_o, h_lse, h_dq, h_dk, h_dv,
     synchronising.  `arena` is a uint8 CUDA tensor of at least psa_step_host_arena_bytes(plan)
     bytes; nothing is allocated here."""
     import torch
-    for t in (h_q, h_k, h_v, h_do, h_o, h_dq, h_dk, h_dv):
-        assert not t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous()
-    assert not h_lse.is_cuda and h_lse.dtype == torch.float32 and h_lse.is_contiguous()
-    assert arena.is_cuda and arena.dtype == torch.uint8 and arena.is_contiguous()
+    _want_attention(plan, [("h_q", h_q, "q"), ("h_k", h_k, "kv"), ("h_v", h_v, "kv"), ("h_do", h_do, "q"),
+                           ("h_o", h_o, "q"), ("h_dq", h_dq, "q"), ("h_dk", h_dk, "kv"), ("h_dv", h_dv, "kv")],
+                    lse=h_lse, cuda=False)
+    if not (arena.is_cuda and arena.dtype == torch.uint8 and arena.is_contiguous()):
+        raise ValueError("arena must be a contiguous uint8 CUDA tensor")
     _check("psa_step_host",
            load_library().psa_step_host(plan._h, _ptr(h_q), _ptr(h_k), _ptr(h_v), _ptr(h_do), _ptr(h_o), _ptr(h_lse),
                                         _ptr(h_dq), _ptr(h_dk), _ptr(h_dv), _ptr(arena),
@@ -343,6 +410,51 @@ def psa_pack_ffd(unit_len, capacity):
     _check("psa_pack_ffd", load_library().psa_pack_ffd(lens.ctypes.data, len(lens), int(capacity), bins.ctypes.data,
                                                       C.byref(n_bins)))
     return bins[:len(lens)], n_bins.value
+
+
+def psa_pack_ffd_emit(prefix_len, chosen_len, rejected_len, capacity, paired=False):
+    """Packs the units with psa_pack_ffd and lays every pack out for psa_plan.  Returns
+    (bin_of_unit int32 [n], packs) where packs is a list of dicts with the keys cu_seqlens,
+    prefix_len, chosen_len, rejected_len (int32 arrays, ready for psa_plan) and units (the
+    source unit of each sample).  paired=True gives the unshared baseline layout: two samples
+    (P, C, 0), (P, R, 0) per unit.  Host only."""
+    P, Cc, R = _i32(prefix_len), _i32(chosen_len), _i32(rejected_len)
+    n = len(P)
+    m = n * (2 if paired else 1)
+    bins = np.zeros(max(n, 1), dtype=np.int32)
+    off = np.zeros(n + 1, dtype=np.int32)
+    unit, oP, oC, oR = (np.zeros(max(m, 1), dtype=np.int32) for _ in range(4))
+    cu = np.zeros(m + n + 1, dtype=np.int32)
+    n_packs = C.c_int32()
+    _check("psa_pack_ffd_emit", load_library().psa_pack_ffd_emit(
+        P.ctypes.data, Cc.ctypes.data, R.ctypes.data, n, int(capacity), 1 if paired else 0, bins.ctypes.data,
+        C.byref(n_packs), off.ctypes.data, unit.ctypes.data, oP.ctypes.data, oC.ctypes.data, oR.ctypes.data,
+        cu.ctypes.data))
+    packs = []
+    for b in range(n_packs.value):
+        lo, hi = int(off[b]), int(off[b + 1])
+        packs.append({"cu_seqlens": cu[lo + b:hi + b + 1].copy(), "prefix_len": oP[lo:hi].copy(),
+                      "chosen_len": oC[lo:hi].copy(), "rejected_len": oR[lo:hi].copy(), "units": unit[lo:hi].copy()})
+    return bins[:n], packs
+
+
+def psa_logp_labels(token_ids, cu_seqlens, prefix_len, chosen_len, rejected_len):
+    """Label layout of dpo_logp on the shared layout: returns (targets int32 [T], segment_ids
+    int32 [T], fork_rows, fork_targets, fork_segments int32 [n_forks]); response ids 2s = chosen,
+    2s+1 = rejected, -1 = row not scored.  Host only."""
+    tok, cu = _i32(token_ids), _i32(cu_seqlens)
+    P, Cc, R = _i32(prefix_len), _i32(chosen_len), _i32(rejected_len)
+    n, T = len(P), int(cu[-1])
+    if len(cu) != n + 1 or len(tok) < T:
+        raise ValueError("cu_seqlens must have n+1 entries and token_ids at least T entries")
+    targets, seg = np.zeros(max(T, 1), dtype=np.int32), np.zeros(max(T, 1), dtype=np.int32)
+    fr, ft, fs = (np.zeros(max(n, 1), dtype=np.int32) for _ in range(3))
+    nf = C.c_int32()
+    _check("psa_logp_labels", load_library().psa_logp_labels(
+        tok.ctypes.data, cu.ctypes.data, P.ctypes.data, Cc.ctypes.data, R.ctypes.data, n, targets.ctypes.data,
+        seg.ctypes.data, fr.ctypes.data, ft.ctypes.data, fs.ctypes.data, C.byref(nf)))
+    k = nf.value
+    return targets[:T], seg[:T], fr[:k].copy(), ft[:k].copy(), fs[:k].copy()
 
 
 def psa_position_ids(cu_seqlens, prefix_len, chosen_len, rejected_len):

@@ -9,7 +9,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpsa.so")
-SOURCES = ["psa_plan.cpp", "psa_api.cu", "psa_fwd.cu", "psa_bwd.cu", "psa_bwd_static.cu", "dpo_logp.cu", "dpo_loss.cu", "psa_rope.cu"]
+SOURCES = ["psa_plan.cpp", "psa_host_helpers.cpp", "psa_api.cu", "psa_fwd.cu", "psa_bwd.cu", "psa_bwd_static.cu", "psa_selftest.cu",
+           "dpo_logp.cu", "dpo_loss.cu", "psa_rope.cu"]
 
 
 def _stale() -> bool:
@@ -27,9 +28,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
            "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
-    if os.environ.get("PSA_TRACE"):   # debug build: SM-clock timestamps of the first CTA's hand-offs
-        # (read back with psa_trace_dump / psa_trace_dump_fwd, 64 iterations x 16 slots of int64)
-        cmd += ["-DPSA_TRACE"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     res = subprocess.run(cmd, capture_output=True, text=True)

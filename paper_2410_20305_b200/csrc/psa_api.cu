@@ -10,6 +10,15 @@ namespace {
 inline bool misaligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; }
 }  // namespace
 
+namespace psa {
+// The plan's device blob lives on the device that was current when it was uploaded; a launch
+// from another device would hand the kernels pointers that mean nothing there.
+bool plan_on_current_device(const psa_plan_t* plan) {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess && dev == plan->device;
+}
+}  // namespace psa
+
 extern "C" psa_status_t psa_fwd(const psa_plan_t* plan, const void* q, const void* k, const void* v, void* o,
                                 float* lse, int32_t* device_status, void* stream) {
   if (!plan) return PSA_ERR_INVALID_ARG;
@@ -18,6 +27,7 @@ extern "C" psa_status_t psa_fwd(const psa_plan_t* plan, const void* q, const voi
   if (!q || !k || !v || !o || !lse) return PSA_ERR_INVALID_ARG;
   if (misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(o, 16) || misaligned(lse, 4))
     return PSA_ERR_ALIGNMENT;
+  if (!psa::plan_on_current_device(plan)) return PSA_ERR_INVALID_ARG;
   psa::note_plan_use(plan, stream);
   return psa::launch_fwd(plan, q, k, v, o, lse, device_status, stream);
 }
@@ -33,8 +43,25 @@ extern "C" psa_status_t psa_bwd(const psa_plan_t* plan, const void* d_o, const v
       misaligned(dq, 16) || misaligned(dk, 16) || misaligned(dv, 16) || misaligned(lse, 4) ||
       misaligned(workspace, 256))
     return PSA_ERR_ALIGNMENT;
+  if (!psa::plan_on_current_device(plan)) return PSA_ERR_INVALID_ARG;
   psa::note_plan_use(plan, stream);
-  return psa::launch_bwd(plan, d_o, q, k, v, o, lse, dq, dk, dv, workspace, device_status, stream);
+  return psa::launch_bwd(plan, d_o, q, k, v, o, lse, dq, dk, dv, workspace, false, device_status, stream);
+}
+
+extern "C" psa_status_t psa_bwd_f32(const psa_plan_t* plan, const void* d_o, const void* q, const void* k,
+                                    const void* v, const void* o, const float* lse, float* dq, float* dk,
+                                    float* dv, void* workspace, int32_t* device_status, void* stream) {
+  if (!plan) return PSA_ERR_INVALID_ARG;
+  if (plan->T == 0) return PSA_OK;
+  if (!plan->d_blob) return PSA_ERR_INVALID_ARG;
+  if (!d_o || !q || !k || !v || !o || !lse || !dq || !dk || !dv || !workspace) return PSA_ERR_INVALID_ARG;
+  if (misaligned(d_o, 16) || misaligned(q, 16) || misaligned(k, 16) || misaligned(v, 16) || misaligned(o, 16) ||
+      misaligned(dq, 16) || misaligned(dk, 16) || misaligned(dv, 16) || misaligned(lse, 4) ||
+      misaligned(workspace, 256))
+    return PSA_ERR_ALIGNMENT;
+  if (!psa::plan_on_current_device(plan)) return PSA_ERR_INVALID_ARG;
+  psa::note_plan_use(plan, stream);
+  return psa::launch_bwd(plan, d_o, q, k, v, o, lse, dq, dk, dv, workspace, true, device_status, stream);
 }
 
 namespace {
@@ -72,6 +99,7 @@ extern "C" psa_status_t psa_step_host(const psa_plan_t* plan, const void* h_q, c
   const StepArena a = step_arena_layout(plan);
   if (arena_bytes < a.bytes) return PSA_ERR_INVALID_ARG;
   if (misaligned(arena, 256)) return PSA_ERR_ALIGNMENT;
+  if (!psa::plan_on_current_device(plan)) return PSA_ERR_INVALID_ARG;
   psa::note_plan_use(plan, stream);
   char* base = static_cast<char*>(arena);
   const cudaStream_t st = cudaStream_t(stream);
@@ -91,7 +119,7 @@ extern "C" psa_status_t psa_step_host(const psa_plan_t* plan, const void* h_q, c
     return psa::check_last_cuda_error("psa_step_host copy out");
   rc = psa::launch_bwd(plan, base + a.d_o, base + a.q, base + a.k, base + a.v, base + a.o,
                        reinterpret_cast<const float*>(base + a.lse), base + a.dq, base + a.dk, base + a.dv,
-                       base + a.ws, device_status, stream);
+                       base + a.ws, false, device_status, stream);
   if (rc != PSA_OK) return rc;
   if (!copy(h_dq, base + a.dq, nq, cudaMemcpyDeviceToHost) || !copy(h_dk, base + a.dk, nk, cudaMemcpyDeviceToHost) ||
       !copy(h_dv, base + a.dv, nk, cudaMemcpyDeviceToHost))

@@ -36,12 +36,6 @@
 #include "psa_tensormap.h"
 
 namespace psa {
-#ifdef PSA_TRACE
-__device__ long long g_psa_trace[64 * 16];
-__device__ long long g_psa_cta_trace[4096 * 4];   // per CTA: start, end (globaltimer ns), SM id, iterations
-__device__ long long g_psa_cta_phase[4096 * 8];   // per CTA: globaltimer at a few points of its life
-#define PSA_CTA_PHASE(k) do { if (blockIdx.x < 4096) { unsigned long long t_; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_)); g_psa_cta_phase[blockIdx.x * 8 + (k)] = (long long)t_; } } while (0)
-#endif
 namespace {
 
 using namespace dev;
@@ -58,10 +52,11 @@ struct BwdParams {
   const float* lse;         // [Hq, T]
   const float* delta;       // [Hq, T]
   float* dq_accum;          // [T, Hq, D] fp32
-  __nv_bfloat16* dk;
-  __nv_bfloat16* dv;
+  void* dk;                 // [T, Hkv, D], bf16 or (f32_out) fp32
+  void* dv;
   int32_t* status;
   int32_t T, Hq, Hkv;
+  int32_t f32_out;          // gradients leave as fp32: dk, dv from the accumulators, dq = dq_accum
   float scale, scale_log2;
 };
 
@@ -93,17 +88,6 @@ enum {
   B_S_FULL, B_DP_FULL, B_P_FULL, B_DS_FULL, B_DS_EMPTY, B_DQ_FULL, B_DQ_EMPTY, B_DONE, B_COUNT
 };
 
-// Debug builds (-DPSA_TRACE) record SM-clock timestamps of the first CTA's hand-offs.
-#ifdef PSA_TRACE
-#define PSA_TRACE_MARK(it, slot)                                                        \
-  do {                                                                                  \
-    if (blockIdx.x == 0 && (it) < 64) g_psa_trace[(it) * 16 + (slot)] = clock64();       \
-  } while (0)
-#else
-#define PSA_CTA_PHASE(k) do {} while (0)
-#define PSA_TRACE_MARK(it, slot) do {} while (0)
-#endif
-
 
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
@@ -125,15 +109,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   float* s_delta = reinterpret_cast<float*>(smem_raw + L::kDelta);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#ifdef PSA_TRACE
-  if (threadIdx.x == 0 && blockIdx.x < 4096) {
-    unsigned long long t; unsigned sm;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
-    g_psa_cta_trace[blockIdx.x * 4 + 0] = (long long)t;
-    g_psa_cta_trace[blockIdx.x * 4 + 2] = sm;
-  }
-#endif
   const int tile_idx = prm.cta_map[2 * blockIdx.x];
   const int hk = prm.cta_map[2 * blockIdx.x + 1];
   const int g = prm.Hq / prm.Hkv;
@@ -141,7 +116,7 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const int32_t* ent = prm.entries + rec.list_off;
   const int n_list = rec.list_cnt;
   const int n_it = n_list * g;
-  const WaitCtx wctx{abort_flag, prm.status};
+  const WaitCtx wctx{abort_flag, prm.status, kWaitLimitClocks};
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -180,7 +155,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  if (threadIdx.x == 0) PSA_CTA_PHASE(0);
 
   // Iteration it -> (query head of the group, entry of the list).
   auto head_of = [&](int it) { return hk * g + it / n_list; };
@@ -204,7 +178,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         mbar_expect_tx(bar(B_Q_FULL0 + st), L::kTileBytes);
         for (int s = 0; s < L::kSub; ++s) tma_load_3d(sQ(st) + s * L::kSubBytes, &tm_q, s * 64, h, qrow, bar(B_Q_FULL0 + st));
         mbar_wait(bar(B_DO_EMPTY), (it - 1) & 1, wctx);   // dV of the previous iteration has read dO
-        PSA_TRACE_MARK(it, 11);
         mbar_expect_tx(bar(B_DO_FULL), L::kTileBytes);
         for (int s = 0; s < L::kSub; ++s) tma_load_3d(sDO + s * L::kSubBytes, &tm_do, s * 64, h, qrow, bar(B_DO_FULL));
       }
@@ -235,7 +208,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int st = it & 1, ph = (it >> 1) & 1;
         mbar_wait(bar(B_Q_FULL0 + st), ph, wctx);
         tc_fence_after();
-        PSA_TRACE_MARK(it, 0);
         const uint32_t q_lo = st ? q1_k : q0_k;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
@@ -252,12 +224,9 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // dP^T = V dO^T into the columns the previous dQ occupied: wait until it was read out.
         // (This commit also covers the previous iteration's dK / dQ products, so a completed
         // dP^T tells the compute warps that the dS buffer is free again.)
-        PSA_TRACE_MARK(it, 13);
         mbar_wait(bar(B_DO_FULL), it & 1, wctx);
-        PSA_TRACE_MARK(it, 14);
         if (it > 0) mbar_wait(bar(B_DQ_EMPTY), (it - 1) & 1, wctx);
         tc_fence_after();
-        PSA_TRACE_MARK(it, 1);
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = ((kk >> 2) * L::kSubBytes + (kk & 3) * 32) >> 4;
@@ -267,7 +236,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // dV += P^T dO   (reduction over the 128 query rows, 16 per instruction)
         mbar_wait(bar(B_P_FULL), it & 1, wctx);
         tc_fence_after();
-        PSA_TRACE_MARK(it, 2);
         // P^T of query columns [64 h, 64 h + 64) sits in S-region columns [64 h, 64 h + 32), the
         // second term of a PRECISE tile in [64 h + 32, 64 h + 64); 16 queries = 8 columns.
         for (int term = 0; term < n_terms; ++term) {
@@ -277,7 +245,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                        do_mn + kk * (2048 >> 4), idesc_dv, (it > 0) || (kk > 0) || (term > 0), issuer);
         }
         umma_commit_w(bar(B_DO_EMPTY), issuer);
-        PSA_TRACE_MARK(it, 15);
         // The next S^T goes in now, so that the compute warps can start on it while the dK / dQ
         // products of this iteration run.
         if (it + 1 < n_it) issue_s(it + 1);
@@ -288,7 +255,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         mbar_wait(bar(B_DS_FULL), ds_ph, wctx);
         ds_ph ^= 1;
         tc_fence_after();
-        PSA_TRACE_MARK(it, 3);
         for (int term = 0; term < n_terms; ++term) {
 #pragma unroll
           for (int kk = 0; kk < kTile / 16; ++kk)
@@ -309,7 +275,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                        (kk > 0) || (term > 0), issuer);
         }
         umma_commit_w(bar(B_DQ_FULL), issuer);
-        PSA_TRACE_MARK(it, 4);
       }
       umma_commit_w(bar(B_DONE), issuer);   // every product, the last dK included, has completed
     }
@@ -364,14 +329,10 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
       mbar_wait(bar(B_S_FULL), it & 1, wctx);
       tc_fence_after();
-      if (leader) PSA_TRACE_MARK(it, 5);
-      if (leader && it == 0) PSA_CTA_PHASE(1);
-      if (leader && it == 1) PSA_CTA_PHASE(6);
       float p[64];
       {
         uint32_t sv[64];   // both loads in flight, one wait
         tmem_ld64_wait(tmem + lane_base + kColS + c0, sv);
-        if (leader) PSA_TRACE_MARK(it, 12);
         const float4* l4 = reinterpret_cast<const float4*>(s_lse + st * kTile + c0);
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
@@ -406,13 +367,11 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar(B_P_FULL));
-      if (leader) PSA_TRACE_MARK(it, 6);
 
       // dS^T = P^T * (dP^T - delta) -> shared memory.  The buffer is free: dP^T of this
       // iteration was issued, and so completed, after the previous iteration's dK / dQ products.
       mbar_wait(bar(B_DP_FULL), it & 1, wctx);
       tc_fence_after();
-      if (leader) PSA_TRACE_MARK(it, 7);
       if constexpr (kPrecise) {
         if ((e >> 2) == 0) {
           // Rows of a sample's first query tile see only this key tile, and they are the rows
@@ -490,7 +449,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       fence_proxy_async_smem();
       tc_fence_before();
       mbar_arrive(bar(B_DS_FULL));
-      if (leader) PSA_TRACE_MARK(it, 8);
       if constexpr (kPrecise) {
         // second term: same buffer, once the products of the first term have read it
         mbar_wait(bar(B_DS_EMPTY), dse_ph, wctx);
@@ -515,13 +473,31 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (entry_of(it) & 2) iteration(it, std::true_type{});
       else iteration(it, std::false_type{});
     }
-    if (leader) PSA_CTA_PHASE(2);
     mbar_wait(bar(B_DONE), 0, wctx);
     tc_fence_after();
-    if (leader) PSA_CTA_PHASE(3);
 
-    // ---- epilogue: this half's columns of dV and dK (scaled) -> bf16
-    if (rec.len - rec.local0 >= kTile) {
+    // ---- epilogue: this half's columns of dV and dK (scaled) -> bf16, or fp32 as they are
+    if (prm.f32_out) {
+      // fp32 outputs: the accumulators leave unrounded, one row per thread.
+      const int64_t row = int64_t(rec.row0) + r;
+#pragma unroll
+      for (int which = 0; which < 2; ++which) {
+        const float mul = which ? prm.scale : 1.f;
+        float* dst_row = static_cast<float*>(which ? prm.dk : prm.dv) + (row * prm.Hkv + hk) * D + half * DH;
+#pragma unroll
+        for (int ch = 0; ch < DH / 32; ++ch) {
+          uint32_t v[32];
+          tmem_ld32_wait(tmem + lane_base + (which ? kColDK : kColDV) + half * DH + ch * 32, v);
+          if (kv_valid) {
+            float4* dst = reinterpret_cast<float4*>(dst_row + ch * 32);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              dst[i] = make_float4(__uint_as_float(v[4 * i + 0]) * mul, __uint_as_float(v[4 * i + 1]) * mul,
+                                   __uint_as_float(v[4 * i + 2]) * mul, __uint_as_float(v[4 * i + 3]) * mul);
+          }
+        }
+      }
+    } else if (rec.len - rec.local0 >= kTile) {
       // Full tile: rows go through shared memory (the K and V buffers are free now) in the
       // 128-byte-swizzled layout of the tensor maps, and two TMA stores per tensor write them
       // out coalesced.  (A ragged last tile must not touch the rows of the next sample, which the
@@ -560,8 +536,8 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
     } else {
     const int64_t row = int64_t(rec.row0) + r;
-    __nv_bfloat16* dv_row = prm.dv + (row * prm.Hkv + hk) * D + half * DH;
-    __nv_bfloat16* dk_row = prm.dk + (row * prm.Hkv + hk) * D + half * DH;
+    __nv_bfloat16* dv_row = static_cast<__nv_bfloat16*>(prm.dv) + (row * prm.Hkv + hk) * D + half * DH;
+    __nv_bfloat16* dk_row = static_cast<__nv_bfloat16*>(prm.dk) + (row * prm.Hkv + hk) * D + half * DH;
 #pragma unroll
     for (int which = 0; which < 2; ++which) {
       const float mul = which ? prm.scale : 1.f;
@@ -599,7 +575,6 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int h = head_of(it);
       mbar_wait(bar(B_DQ_FULL), it & 1, wctx);
       tc_fence_after();
-      if (leader) PSA_TRACE_MARK(it, 9);
       // Pull the whole row out of TMEM first and release the columns at once: the next dP^T
       // is waiting for them.  Staging and reducing then proceed from registers, at the pace
       // the reduce-adds are absorbed by L2.
@@ -634,28 +609,17 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           tma_commit_group();
         }
       }
-      if (leader) PSA_TRACE_MARK(it, 10);
     }
     if (leader) tma_wait_group_read<0>();   // shared memory must outlive the last reduce's reads (the adds
                                             // themselves complete before the kernel does)
-    if (leader) PSA_CTA_PHASE(5);
   }
 
-  if (threadIdx.x == 128) PSA_CTA_PHASE(4);   // first worker: its epilogue stores are issued
   tc_fence_before();
   __syncthreads();
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem, kBwdTmemCols);
   }
-#ifdef PSA_TRACE
-  if (threadIdx.x == 0 && blockIdx.x < 4096) {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    g_psa_cta_trace[blockIdx.x * 4 + 1] = (long long)t;
-    g_psa_cta_trace[blockIdx.x * 4 + 3] = n_it;
-  }
-#endif
 }
 
 // delta[h][t] = sum_c dO[t,h,c] * O[t,h,c]; one 16-byte load per thread and tensor.  The kernel also
@@ -754,18 +718,20 @@ psa_bwd_convert_kernel(const float4* __restrict__ acc, uint2* __restrict__ dq, i
 template <int D>
 psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q, const void* k, const void* v,
                           const void* o, const float* lse, void* dq, void* dk, void* dv, void* workspace,
-                          int32_t* device_status, cudaStream_t stream) {
+                          bool f32_out, int32_t* device_status, cudaStream_t stream) {
   using L = BwdSmem<D>;
   const int64_t T = plan->T;
   const BwdWorkspace ws = bwd_workspace_layout(T, plan->Hq, D);
   char* wsp = static_cast<char*>(workspace);
-  float* dq_accum = reinterpret_cast<float*>(wsp + ws.dq_accum_off);
+  // With fp32 outputs the caller's dq is the accumulator itself and nothing is converted.
+  float* dq_accum = f32_out ? static_cast<float*>(dq) : reinterpret_cast<float*>(wsp + ws.dq_accum_off);
   float* delta = reinterpret_cast<float*>(wsp + ws.delta_off);
 
   CUtensorMap tm_q, tm_k, tm_v, tm_do, tm_dq, tm_dk, tm_dv;
   if (!make_tile_map_bf16(&tm_q, q, T, plan->Hq, D) || !make_tile_map_bf16(&tm_k, k, T, plan->Hkv, D) ||
       !make_tile_map_bf16(&tm_v, v, T, plan->Hkv, D) || !make_tile_map_bf16(&tm_do, d_o, T, plan->Hq, D) ||
       !make_tile_map(&tm_dq, dq_accum, T, plan->Hq, D, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, 32, 128) ||
+      // (with fp32 outputs dk and dv leave through per-thread stores; their maps are built but not used)
       !make_tile_map_bf16(&tm_dk, dk, T, plan->Hkv, D) || !make_tile_map_bf16(&tm_dv, dv, T, plan->Hkv, D))
     return PSA_ERR_CUDA;
   if (cudaFuncSetAttribute(psa_bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kRequest) != cudaSuccess)
@@ -790,8 +756,9 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
   prm.lse = lse;
   prm.delta = delta;
   prm.dq_accum = dq_accum;
-  prm.dk = static_cast<__nv_bfloat16*>(dk);
-  prm.dv = static_cast<__nv_bfloat16*>(dv);
+  prm.dk = dk;
+  prm.dv = dv;
+  prm.f32_out = f32_out ? 1 : 0;
   prm.status = device_status;
   prm.T = plan->T;
   prm.Hq = plan->Hq;
@@ -803,7 +770,7 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
     ProfileScope prof(1, stream);
     psa_bwd_kernel<D><<<grid, kBwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_dq, tm_dk, tm_dv, prm);
   }
-  {
+  if (!f32_out) {
     const int64_t n_vec4 = n_rows * D / 4;
     psa_bwd_convert_kernel<<<unsigned((n_vec4 + 255) / 256), 256, 0, stream>>>(
         reinterpret_cast<const float4*>(dq_accum), static_cast<uint2*>(dq), n_vec4);
@@ -815,23 +782,13 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
 
 psa_status_t launch_bwd(const psa_plan_t* plan, const void* d_o, const void* q, const void* k, const void* v,
                         const void* o, const float* lse, void* dq, void* dk, void* dv, void* workspace,
-                        int32_t* device_status, void* stream) {
+                        bool f32_out, int32_t* device_status, void* stream) {
   if (plan->d == 128)
-    return launch_bwd_t<128>(plan, d_o, q, k, v, o, lse, dq, dk, dv, workspace, device_status, cudaStream_t(stream));
-  return launch_bwd_t<64>(plan, d_o, q, k, v, o, lse, dq, dk, dv, workspace, device_status, cudaStream_t(stream));
+    return launch_bwd_t<128>(plan, d_o, q, k, v, o, lse, dq, dk, dv, workspace, f32_out, device_status,
+                             cudaStream_t(stream));
+  return launch_bwd_t<64>(plan, d_o, q, k, v, o, lse, dq, dk, dv, workspace, f32_out, device_status,
+                          cudaStream_t(stream));
 }
 
 }  // namespace psa
 
-#ifdef PSA_TRACE
-// Debug builds only: copies the 64 x 16 timestamp table of the last psa_bwd launch to the host.
-extern "C" int psa_trace_dump_phases(long long* host_out) {
-  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_cta_phase, sizeof(long long) * 4096 * 8));
-}
-extern "C" int psa_trace_dump_ctas(long long* host_out) {
-  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_cta_trace, sizeof(long long) * 4096 * 4));
-}
-extern "C" int psa_trace_dump(long long* host_out) {
-  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_trace, sizeof(long long) * 64 * 16));
-}
-#endif

@@ -62,11 +62,13 @@ extern "C" psa_status_t psa_bwd_static_scratch(const psa_plan_t* plan, const voi
                    plan->bwd_workspace_bytes, kStaticScratchBytes);
     return PSA_ERR_UNSUPPORTED;
   }
+  // The plan's tile map and the scratch array must be on the same device as the launch.
+  if (!psa::plan_on_current_device(plan)) return PSA_ERR_INVALID_ARG;
   void* scratch = nullptr;
   const psa_status_t st = static_scratch_address(&scratch);
   if (st != PSA_OK) return st;
   // launch_bwd clears the dq accumulator itself (it must start at zero) and overwrites delta,
   // so whatever the previous call left in the array does not matter.
   psa::note_plan_use(plan, stream);
-  return psa::launch_bwd(plan, d_o, q, k, v, o, lse, dq, dk, dv, scratch, device_status, stream);
+  return psa::launch_bwd(plan, d_o, q, k, v, o, lse, dq, dk, dv, scratch, false, device_status, stream);
 }

@@ -47,14 +47,17 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 
-// Shared by all threads of a CTA: abort flag (shared memory) + status word (global, may be null).
+// Shared by all threads of a CTA: abort flag (shared memory), status word (global, may be null)
+// and the number of SM clocks after which a wait gives up.
+constexpr long long kWaitLimitClocks = 4000000000LL;   // about two seconds: the product kernels' limit
 struct WaitCtx {
   volatile int* abort_flag;
   int32_t* status;
+  long long limit_clocks;
 };
 
 // Bounded wait for the phase with the given parity to complete.  Gives up after
-// about two seconds of SM clock, or at once when another wait of this CTA already gave up.
+// ctx.limit_clocks SM clocks, or at once when another wait of this CTA already gave up.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& ctx) {
   if (mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
@@ -62,7 +65,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const W
     if (mbar_try_wait(bar, parity)) return;
     if ((spins & 63u) == 0u) {
       if (*ctx.abort_flag) return;
-      if (clock64() - t0 > 4000000000LL) {
+      if (clock64() - t0 > ctx.limit_clocks) {
         *ctx.abort_flag = 1;
         if (ctx.status) atomicOr(ctx.status, PSA_DEVSTAT_WAIT_EXPIRED);
         return;

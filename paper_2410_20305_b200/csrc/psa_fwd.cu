@@ -29,27 +29,6 @@
 #include "psa_tensormap.h"
 
 namespace psa {
-// Debug builds (-DPSA_TRACE) record SM-clock timestamps of the first CTA's hand-offs.
-#ifdef PSA_TRACE
-__device__ long long g_psa_trace_fwd[64 * 16];
-__device__ long long g_psa_cta_trace_fwd[8192 * 4];   // per CTA: start, end (globaltimer ns), SM id, iterations
-#define PSA_FWD_MARK(it, slot)                                                            \
-  do {                                                                                    \
-    if (blockIdx.x == 0 && (it) < 64) g_psa_trace_fwd[(it) * 16 + (slot)] = clock64();     \
-  } while (0)
-__device__ long long g_psa_cta_phase_fwd[8192 * 8];   // per CTA: globaltimer at eight points of its life
-#define PSA_FWD_PHASE(slot)                                                               \
-  do {                                                                                    \
-    if (blockIdx.x < 8192) {                                                              \
-      unsigned long long t_;                                                              \
-      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_));                               \
-      g_psa_cta_phase_fwd[blockIdx.x * 8 + (slot)] = (long long)t_;                       \
-    }                                                                                     \
-  } while (0)
-#else
-#define PSA_FWD_MARK(it, slot) do {} while (0)
-#define PSA_FWD_PHASE(slot) do {} while (0)
-#endif
 namespace {
 
 using namespace dev;
@@ -119,22 +98,13 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + L::kAbort);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-#ifdef PSA_TRACE
-  if (threadIdx.x == 0 && blockIdx.x < 8192) {
-    unsigned long long t; unsigned sm;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
-    g_psa_cta_trace_fwd[blockIdx.x * 4 + 0] = (long long)t;
-    g_psa_cta_trace_fwd[blockIdx.x * 4 + 2] = sm;
-  }
-#endif
   // The CTA's work items: 2 b and 2 b + 1 of the list (longest first, so the CTAs stay sorted by length and the
   // short ones still fill the tail of the launch); the last CTA of an odd count has one item.
   const int idx0 = 2 * int(blockIdx.x), idx1 = idx0 + 1;
   const int n_items = idx1 < prm.n_items ? 2 : 1;
   FwdItem* s_item = reinterpret_cast<FwdItem*>(gen_base + L::kItems);
   int32_t* s_ent_all = reinterpret_cast<int32_t*>(gen_base + L::kEnt);
-  const WaitCtx wctx{abort_flag, prm.status};
+  const WaitCtx wctx{abort_flag, prm.status, kWaitLimitClocks};
   // Every role reads the list entry of every iteration: the head of each item's list is kept in shared memory.
   struct ItemView {
     TileRec rec;
@@ -200,7 +170,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  if (threadIdx.x == 128) PSA_FWD_PHASE(1);
 
   if (warp < 4) {
    setmaxnreg_dec<kRegsWg0>();
@@ -245,9 +214,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const ItemView w = view(item);
       mbar_wait(bar(BAR_Q_FULL), item & 1, wctx);
       for (int it = 0; it < w.n_it; ++it, ++g) {
-        PSA_FWD_MARK(it, 0);
         mbar_wait(bar(BAR_K_FULL), g & 1, wctx);
-        PSA_FWD_MARK(it, 1);
         // The S columns are also where P_{it-1} lives.  UMMAs issued by one thread execute in
         // issue order, so this S = Q K^T cannot overwrite P before the previous P V has read it.
         tc_fence_after();
@@ -258,11 +225,8 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         umma_commit_w(bar(BAR_K_EMPTY), issuer);
         umma_commit_w(bar(BAR_S_FULL), issuer);
-        PSA_FWD_MARK(it, 2);
         mbar_wait(bar(BAR_V_FULL), g & 1, wctx);
-        PSA_FWD_MARK(it, 3);
         mbar_wait(bar(BAR_P_FULL), g & 1, wctx);
-        PSA_FWD_MARK(it, 4);
         tc_fence_after();
         // P of key half hf lies in columns [64 hf, 64 hf + 32) of the S region (two bf16 per column);
         // PRECISE tiles carry a second bf16 term in columns [64 hf + 32, 64 hf + 64).
@@ -277,7 +241,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         umma_commit_w(bar(BAR_V_EMPTY), issuer);
         umma_commit_w(bar(BAR_O_FULL), issuer);
-        PSA_FWD_MARK(it, 5);
       }
       }
     }
@@ -320,9 +283,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const bool precise = (e & 2) != 0;
       mbar_wait(bar(BAR_S_FULL), g & 1, wctx);
       tc_fence_after();
-      if (threadIdx.x == 128) PSA_FWD_MARK(it, 6);
-      if (threadIdx.x == 128 && it == 0) PSA_FWD_PHASE(2);
-      if (threadIdx.x == 128 && it == 1) PSA_FWD_PHASE(3);
       // Allowed keys of this row in a PARTIAL tile, relative to the tile: [0, a) and [b, b + span).
       int a = kTile, b = 0;
       uint32_t span = 0;
@@ -409,7 +369,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(bar(BAR_P_FULL));
-        if (threadIdx.x == 128) PSA_FWD_MARK(it, 9);
         continue;
       }
       if (it > 0 && !precise) {
@@ -485,7 +444,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           tc_wait_st();
           tc_fence_before();
           mbar_arrive(bar(BAR_P_FULL));
-          if (threadIdx.x == 128) PSA_FWD_MARK(it, 9);
           fast_done = true;
         }
       }
@@ -529,7 +487,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         pair_sync();
         mx = fmaxf(mx, slot[(hfz ^ 1) * kTile + r]);
       }
-      if (threadIdx.x == 128) PSA_FWD_MARK(it, 7);
       const float m_new = fmaxf(m_run, mx);
       // Keep a stale maximum while it is within 2^8 of the true one: P stays <= 256
       // and the accumulator needs no rescaling.  (-inf) - (-inf) is NaN -> false.
@@ -555,7 +512,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           tmem_st32(tmem + lane_base + col, v);
         }
       }
-      if (threadIdx.x == 128) PSA_FWD_MARK(it, 8);
       const float mc = (m_run == -INFINITY) ? 0.f : m_run * c;
       float s4[4] = {0.f, 0.f, 0.f, 0.f};
       uint64_t sum2[2] = {0ull, 0ull};                 // two packed pairs of partial row sums
@@ -627,10 +583,8 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar(BAR_P_FULL));
-      if (threadIdx.x == 128) PSA_FWD_MARK(it, 9);
     }
 
-    if (threadIdx.x == 128) PSA_FWD_PHASE(4);
     // ---- epilogue: O / l -> bf16, lse.  The two halves of the row sum meet in shared memory.
     {
       float* slot = xchg + (xs & 1) * 2 * kTile;
@@ -643,7 +597,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_wait(bar(BAR_O_FULL), (gbase + n_it - 1) & 1, wctx);
       tc_fence_after();
     }
-    if (threadIdx.x == 128) PSA_FWD_PHASE(5);
     const float inv_l = 1.f / l_run;
     const int64_t row = int64_t(rec.row0) + r;
     __nv_bfloat16* orow = prm.o + (row * prm.Hq + h) * D + hfz * (D / 2);
@@ -698,7 +651,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (threadIdx.x == 128 && item == 0) mbar_arrive(bar(BAR_STAGE_FREE));
     gbase += n_it;
     }   // items
-    if (threadIdx.x == 128) PSA_FWD_PHASE(6);
   }
 
   tc_fence_before();
@@ -707,14 +659,6 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
   }
-#ifdef PSA_TRACE
-  if (threadIdx.x == 0 && blockIdx.x < 8192) {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    g_psa_cta_trace_fwd[blockIdx.x * 4 + 1] = (long long)t;
-    g_psa_cta_trace_fwd[blockIdx.x * 4 + 3] = n_it;
-  }
-#endif
 }
 
 template <int D>
@@ -756,14 +700,3 @@ psa_status_t launch_fwd(const psa_plan_t* plan, const void* q, const void* k, co
 
 }  // namespace psa
 
-#ifdef PSA_TRACE
-extern "C" int psa_trace_dump_ctas_fwd(long long* host_out) {
-  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_cta_trace_fwd, sizeof(long long) * 8192 * 4));
-}
-extern "C" int psa_trace_dump_phases_fwd(long long* host_out) {
-  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_cta_phase_fwd, sizeof(long long) * 8192 * 8));
-}
-extern "C" int psa_trace_dump_fwd(long long* host_out) {
-  return int(cudaMemcpyFromSymbol(host_out, psa::g_psa_trace_fwd, sizeof(long long) * 64 * 16));
-}
-#endif

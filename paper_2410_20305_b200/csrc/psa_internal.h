@@ -72,6 +72,9 @@ namespace psa {
 // other than the upload's is used, makes it wait for the upload (which is asynchronous).
 void note_plan_use(const psa_plan_t* plan, void* stream);
 
+// True when the current CUDA device is the one the plan's device blob was uploaded to.
+bool plan_on_current_device(const psa_plan_t* plan);
+
 // Returns PSA_OK if no CUDA error is pending, else PSA_ERR_CUDA; with PSA_DEBUG set in the
 // environment the CUDA error string is written to stderr.
 psa_status_t check_last_cuda_error(const char* where);
@@ -97,5 +100,5 @@ psa_status_t launch_fwd(const psa_plan_t* plan, const void* q, const void* k, co
                         float* lse, int32_t* device_status, void* stream);
 psa_status_t launch_bwd(const psa_plan_t* plan, const void* d_o, const void* q, const void* k,
                         const void* v, const void* o, const float* lse, void* dq, void* dk, void* dv,
-                        void* workspace, int32_t* device_status, void* stream);
+                        void* workspace, bool f32_out, int32_t* device_status, void* stream);
 }  // namespace psa

@@ -65,6 +65,24 @@ def test_brute_force_python_loops():
             assert bool(got[q, kv]) == want, (q, kv)
 
 
+def test_row_interval_form():
+    """A different statement of the same mask, from the sample boundaries alone: a prompt or
+    chosen row q sees the keys [sample start, q]; a rejected row sees the prompt
+    [sample start, chosen start) and its own response [rejected start, q]."""
+    pack = wl.random_pack(17, 4, 14, 1, 1, 8)
+    got = orc.packed_mask(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len)
+    want = np.zeros_like(got)
+    for s in range(pack.n_samples):
+        ds = int(pack.cu_seqlens[s]); cs = ds + int(pack.prefix_len[s]); rs = cs + int(pack.chosen_len[s])
+        for q in range(ds, int(pack.cu_seqlens[s + 1])):
+            if q < rs:
+                want[q, ds:q + 1] = True
+            else:
+                want[q, ds:cs] = True
+                want[q, rs:q + 1] = True
+    assert (got == want).all()
+
+
 def test_tiny_mask_count_matches_closed_form():
     rows = _load("tiny_mask_count.txt")
     pack = wl.config_pack(0)
