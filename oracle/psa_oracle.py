@@ -26,6 +26,11 @@ Paper passages each function follows:
   from the packed row with the response boundaries (Section 3.2).
 * ``ideal_token_speedup`` / ``ideal_attention_speedup``: the two footnotes of
   Section 4.2 (2(p+c)/(p+2c) and 2(p+c)^2/(2(p+c)^2-p^2)).
+* ``ffd_pack`` / ``ffd_pack_layout``: Section 3.2 and Section 4.3.2 (first-fit-decreasing
+  packing of prompt-plus-both-responses units; the lay-out of every pack).
+* ``attention_layer_fwd`` / ``attention_layer_bwd``: the full attention layer of the
+  Section 4.2 micro-benchmark (projections, rotary embedding on the shared layout's
+  position ids of Section 3.1, attention, output projection) and its gradient.
 * ``dpo_loss`` / ``dpo_logp_grad``: Eq. 1 (Section 2.1).  The equation is printed as a
   ratio of logs; it is read as the DPO loss of its cited source,
   -log sigmoid(beta * [(lp_theta(chosen) - lp_ref(chosen)) - (lp_theta(rejected) - lp_ref(rejected))]),
@@ -435,6 +440,31 @@ def ffd_pack(unit_lengths, capacity):
     return bin_of
 
 
+def ffd_pack_layout(prefix_len, chosen_len, rejected_len, capacity, paired=False):
+    """The packs a first-fit-decreasing sampler hands to the attention layers (Section 3.2: the
+    packing unit is the prompt with both responses; Section 4.3.2).  Units are packed by
+    ffd_pack over their lengths, P + C + R in the shared layout and 2P + C + R in the paired
+    baseline layout, where a unit is laid out as two sequences (P, C, 0) and (P, R, 0) next to
+    each other.  Inside a pack the units stand in the order they were placed (longest first,
+    ties by index).  Returns a list of packs, each a dict with cu_seqlens (starting at 0),
+    prefix_len, chosen_len, rejected_len and units (source unit of every sample)."""
+    n = len(prefix_len)
+    unit_len = [(2 if paired else 1) * int(prefix_len[i]) + int(chosen_len[i]) + int(rejected_len[i]) for i in range(n)]
+    bin_of = ffd_pack(unit_len, capacity)
+    packs = [dict(cu_seqlens=[0], prefix_len=[], chosen_len=[], rejected_len=[], units=[])
+             for _ in range(max(bin_of, default=-1) + 1)]
+    for i in sorted(range(n), key=lambda i: (-unit_len[i], i)):
+        pk = packs[bin_of[i]]
+        P, C, R = int(prefix_len[i]), int(chosen_len[i]), int(rejected_len[i])
+        for (p, c, r) in ([(P, C, 0), (P, R, 0)] if paired else [(P, C, R)]):
+            pk["prefix_len"].append(p)
+            pk["chosen_len"].append(c)
+            pk["rejected_len"].append(r)
+            pk["units"].append(i)
+            pk["cu_seqlens"].append(pk["cu_seqlens"][-1] + p + c + r)
+    return packs
+
+
 def optimal_bin_count(unit_lengths, capacity):
     """Fewest bins that hold all units, by exhaustive search (tiny inputs only)."""
     items = sorted((int(x) for x in unit_lengths), reverse=True)
@@ -489,3 +519,45 @@ def rope(x, pos, theta=10000.0):
     cos, sin = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
     x1, x2 = x[..., : d // 2], x[..., d // 2:]
     return np.concatenate([x1 * cos - x2 * sin, x2 * cos + x1 * sin], axis=-1)
+
+
+# --------------------------------------------------------------------------
+# One attention layer on the shared layout (Section 4.2: the full attention-layer benchmark)
+# --------------------------------------------------------------------------
+
+def attention_layer_fwd(x, wq, wk, wv, wo, pos, mask, n_q_heads, n_kv_heads, theta=10000.0, softmax_scale=None):
+    """Query / key / value projections, rotary embedding with the shared layout's position ids,
+    attention under the mask, output projection, all in float64:
+        q = rope(x wq), k = rope(x wk), v = x wv, o = attention(q, k, v), out = o wo.
+    x [T, hidden]; wq [hidden, Hq d]; wk, wv [hidden, Hkv d]; wo [Hq d, hidden].
+    Returns (out [T, hidden], cache) where cache holds what the backward needs."""
+    x, wq, wk, wv, wo = (_as_f64(a) for a in (x, wq, wk, wv, wo))
+    T = x.shape[0]
+    d = wq.shape[1] // n_q_heads
+    q = rope((x @ wq).reshape(T, n_q_heads, d), pos, theta)
+    k = rope((x @ wk).reshape(T, n_kv_heads, d), pos, theta)
+    v = (x @ wv).reshape(T, n_kv_heads, d)
+    o, lse = attention_fwd(q, k, v, mask, softmax_scale)
+    out = o.reshape(T, n_q_heads * d) @ wo
+    return out, dict(q=q, k=k, v=v, o=o, lse=lse)
+
+
+def attention_layer_bwd(x, wq, wk, wv, wo, pos, mask, n_q_heads, n_kv_heads, d_out, theta=10000.0,
+                        softmax_scale=None):
+    """Gradient of sum(out * d_out) for attention_layer_fwd with respect to x and the four weight
+    matrices.  The rotary embedding is a rotation per position, so a gradient passes back
+    through it by the inverse rotation (the same formula with the negated position).
+    Returns dict(dx, dwq, dwk, dwv, dwo)."""
+    x, wq, wk, wv, wo, d_out = (_as_f64(a) for a in (x, wq, wk, wv, wo, d_out))
+    T = x.shape[0]
+    d = wq.shape[1] // n_q_heads
+    out, c = attention_layer_fwd(x, wq, wk, wv, wo, pos, mask, n_q_heads, n_kv_heads, theta, softmax_scale)
+    o2 = c["o"].reshape(T, n_q_heads * d)
+    dwo = o2.T @ d_out
+    d_o = (d_out @ wo.T).reshape(T, n_q_heads, d)
+    dq, dk, dv = attention_bwd(c["q"], c["k"], c["v"], d_o, mask, softmax_scale)
+    neg = -np.asarray(pos, dtype=np.float64)
+    dq2 = rope(dq, neg, theta).reshape(T, -1)
+    dk2 = rope(dk, neg, theta).reshape(T, -1)
+    dv2 = dv.reshape(T, -1)
+    return dict(dx=dq2 @ wq.T + dk2 @ wk.T + dv2 @ wv.T, dwq=x.T @ dq2, dwk=x.T @ dk2, dwv=x.T @ dv2, dwo=dwo)

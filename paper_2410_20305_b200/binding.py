@@ -109,7 +109,7 @@ def _ptr(t):
     return C.c_void_p(0) if t is None else C.c_void_p(t.data_ptr())
 
 
-def _want(t, name, shape, dtype, cuda=True):
+def _want(t, name, shape, dtype, cuda=True, placement=True):
     """Raises ValueError unless tensor `t` has exactly this shape and dtype, is contiguous and
     lives where the call needs it.  The kernels size their tensor maps and grids from the plan
     alone, so a tensor of another pack, or a buffer that is too small, would be read or written
@@ -120,22 +120,23 @@ def _want(t, name, shape, dtype, cuda=True):
         raise ValueError("%s: dtype %s, expected %s" % (name, t.dtype, dtype))
     if not t.is_contiguous():
         raise ValueError("%s must be contiguous" % name)
-    if bool(t.is_cuda) != bool(cuda):
+    if placement and bool(t.is_cuda) != bool(cuda):
         raise ValueError("%s must be a %s tensor" % (name, "CUDA" if cuda else "host"))
 
 
-def _want_attention(plan, bf16, f32=(), lse=None, cuda=True, grads_f32=False):
-    """Shape / dtype checks of the attention tensors against the plan: names in `bf16` are
-    (name, tensor, "q" or "kv") triples."""
+def _want_attention(plan, bf16, f32=(), lse=None, cuda=True):
+    """Checks the attention tensors of a call against the plan: `bf16` and `f32` are lists of
+    (name, tensor, "q" or "kv").  Shapes and dtypes of all of them first, then where they live."""
     import torch
     T, d = plan.total_tokens, plan.head_dim
     heads = {"q": plan.n_q_heads, "kv": plan.n_kv_heads}
-    for name, t, kind in bf16:
-        _want(t, name, (T, heads[kind], d), torch.bfloat16, cuda)
-    for name, t, kind in f32:
-        _want(t, name, (T, heads[kind], d), torch.float32, cuda)
-    if lse is not None:
-        _want(lse, "lse", (plan.n_q_heads, T), torch.float32, cuda)
+    for placement in (False, True):
+        for name, t, kind in bf16:
+            _want(t, name, (T, heads[kind], d), torch.bfloat16, cuda, placement)
+        for name, t, kind in f32:
+            _want(t, name, (T, heads[kind], d), torch.float32, cuda, placement)
+        if lse is not None:
+            _want(lse, "lse", (plan.n_q_heads, T), torch.float32, cuda, placement)
 
 
 class Plan:
@@ -197,12 +198,11 @@ def psa_fwd(plan: Plan, q, k, v, o=None, lse=None, status=None, stream=None):
     """q [T,Hq,d], k, v [T,Hkv,d] bf16 CUDA tensors -> (o [T,Hq,d] bf16, lse [Hq,T] fp32)."""
     import torch
     T = plan.total_tokens
-    _want_attention(plan, [("q", q, "q"), ("k", k, "kv"), ("v", v, "kv")])
     if o is None:
         o = torch.empty_like(q)
     if lse is None:
         lse = torch.empty((plan.n_q_heads, T), dtype=torch.float32, device=q.device)
-    _want_attention(plan, [("o", o, "q")], lse=lse)
+    _want_attention(plan, [("q", q, "q"), ("k", k, "kv"), ("v", v, "kv"), ("o", o, "q")], lse=lse)
     _check("psa_fwd", load_library().psa_fwd(plan._h, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(status),
                                              _stream(stream)))
     return o, lse
@@ -211,14 +211,14 @@ def psa_fwd(plan: Plan, q, k, v, o=None, lse=None, status=None, stream=None):
 def psa_bwd(plan: Plan, d_o, q, k, v, o, lse, dq=None, dk=None, dv=None, workspace=None, status=None, stream=None):
     """Returns (dq [T,Hq,d], dk, dv [T,Hkv,d]) bf16."""
     import torch
-    _want_attention(plan, [("d_o", d_o, "q"), ("q", q, "q"), ("k", k, "kv"), ("v", v, "kv"), ("o", o, "q")], lse=lse)
     if dq is None:
         dq = torch.empty_like(q)
     if dk is None:
         dk = torch.empty_like(k)
     if dv is None:
         dv = torch.empty_like(v)
-    _want_attention(plan, [("dq", dq, "q"), ("dk", dk, "kv"), ("dv", dv, "kv")])
+    _want_attention(plan, [("d_o", d_o, "q"), ("q", q, "q"), ("k", k, "kv"), ("v", v, "kv"), ("o", o, "q"),
+                           ("dq", dq, "q"), ("dk", dk, "kv"), ("dv", dv, "kv")], lse=lse)
     if workspace is None:
         workspace = torch.empty(max(plan.bwd_workspace_bytes, 256), dtype=torch.uint8, device=q.device)
     if not workspace.is_cuda or workspace.numel() * workspace.element_size() < plan.bwd_workspace_bytes:
@@ -233,12 +233,12 @@ def psa_bwd_f32(plan: Plan, d_o, q, k, v, o, lse, dq=None, dk=None, dv=None, wor
     """psa_bwd with fp32 gradient outputs: returns (dq [T,Hq,d], dk, dv [T,Hkv,d]) fp32, the
     kernels' fp32 accumulators written out without the final rounding to bf16."""
     import torch
-    _want_attention(plan, [("d_o", d_o, "q"), ("q", q, "q"), ("k", k, "kv"), ("v", v, "kv"), ("o", o, "q")], lse=lse)
     f32 = lambda t: torch.empty(t.shape, dtype=torch.float32, device=t.device)
     dq = f32(q) if dq is None else dq
     dk = f32(k) if dk is None else dk
     dv = f32(v) if dv is None else dv
-    _want_attention(plan, [], f32=[("dq", dq, "q"), ("dk", dk, "kv"), ("dv", dv, "kv")])
+    _want_attention(plan, [("d_o", d_o, "q"), ("q", q, "q"), ("k", k, "kv"), ("v", v, "kv"), ("o", o, "q")],
+                    f32=[("dq", dq, "q"), ("dk", dk, "kv"), ("dv", dv, "kv")], lse=lse)
     if workspace is None:
         workspace = torch.empty(max(plan.bwd_workspace_bytes, 256), dtype=torch.uint8, device=q.device)
     if not workspace.is_cuda or workspace.numel() * workspace.element_size() < plan.bwd_workspace_bytes:

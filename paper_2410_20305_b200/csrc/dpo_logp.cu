@@ -108,9 +108,12 @@ dpo_logp_kernel(const T* __restrict__ logits, int64_t vocab, int64_t row_stride,
     mx *= kLog2e;
     // One rescale of the running sum per chunk, one exponential per element.
     const float mn = fmaxf(acc.m, mx);
-    float s = acc.s * ex2_approx(acc.m - mn);
+    // A chunk of -inf logits (banned or padded vocabulary entries) before anything finite:
+    // the shift is taken against 0 instead, so that (-inf) - (-inf) never forms; every term is 0.
+    const float sh = (mn == -INFINITY) ? 0.f : mn;
+    float s = acc.s * ex2_approx(acc.m - sh);
 #pragma unroll
-    for (int j = 0; j < kUnroll * E; ++j) s += ex2_approx(fmaf(y[j], kLog2e, -mn));
+    for (int j = 0; j < kUnroll * E; ++j) s += ex2_approx(fmaf(y[j], kLog2e, -sh));
     acc.m = mn;
     acc.s = s;
   }

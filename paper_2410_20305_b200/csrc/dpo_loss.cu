@@ -20,7 +20,6 @@ namespace {
 
 constexpr int kBwdLogpThreads = 1024;   // one CTA per SM: 148 rows (38 MB) in flight, well inside L2
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -231,9 +230,12 @@ dpo_logp_bwd_kernel(const T* __restrict__ logits, int64_t vocab, int64_t row_str
     for (int j = 1; j < E; ++j) mx = fmaxf(mx, y[j]);
     mx *= kLog2e;
     const float mn = fmaxf(acc.m, mx);
-    float s = acc.s * ex2_approx(acc.m - mn);
+    // A chunk of -inf logits (banned or padded vocabulary entries) before anything finite:
+    // the shift is taken against 0 instead, so that (-inf) - (-inf) never forms; every term is 0.
+    const float sh = (mn == -INFINITY) ? 0.f : mn;
+    float s = acc.s * ex2_approx(acc.m - sh);
 #pragma unroll
-    for (int j = 0; j < E; ++j) s += ex2_approx(fmaf(y[j], kLog2e, -mn));
+    for (int j = 0; j < E; ++j) s += ex2_approx(fmaf(y[j], kLog2e, -sh));
     acc.m = mn;
     acc.s = s;
   }

@@ -423,13 +423,15 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
         }
         // The running maximum still holds if no probability of the tile exceeds 2^8 against it.  The
-        // row sum, which is needed anyway, bounds them all: above 256 (or not a number, or a first
-        // contribution to a row whose running maximum is still -inf) the tile goes to the two-pass path.
+        // row sum, which is needed anyway, bounds them all: above 256 (or not a number) the tile goes to
+        // the two-pass path.  So does every tile of a row whose running maximum is still -inf, unless the
+        // whole tile is masked for the warp: exponentials taken against "no maximum yet" may all have
+        // underflowed to 0, which a row sum cannot tell from "nothing to add".
         float a0, a1, b0, b1;
         unpack_f32x2(sum2[0], a0, a1);
         unpack_f32x2(sum2[1], b0, b1);
         const float sumf = (a0 + a1) + (b0 + b1);
-        bool redo = !(sumf <= 256.f) || (m_run == -INFINITY && sumf > 0.f);
+        bool redo = !(sumf <= 256.f) || (m_run == -INFINITY && cls != 0xAu);
         {
           // both threads of a row must take the same path
           float* slot = xchg + (xs & 1) * 2 * kTile;
