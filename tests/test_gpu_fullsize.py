@@ -1,9 +1,12 @@
 """Parity at the full benchmark sizes, in the launch configuration bench.py times.
 
-The dense oracle cannot do a 16k-32k token pack for 32 heads in seconds, so whole samples
-of the pack are checked instead: attention never crosses a sample boundary (the oracle's
-own tests pin that), hence the oracle run on one sample alone, for one kv-head group,
-must reproduce the GPU's outputs on that sample's rows and heads.
+The dense oracle cannot do a 16k-32k token pack for 32 heads in seconds.  Attention never
+crosses a sample boundary (the oracle's own tests pin that), so the oracle is run sample by
+sample: (1) on whole samples for one kv-head group, every element; (2) over the whole pack
+and all heads on sampled outputs it can compute one by one: forward rows of every sample
+(random rows, every prompt / chosen / rejected boundary, tile edges), and on the longest
+sample, where the tile lists are longest, gradients of sampled query rows and of key
+positions in the tails of the responses (the oracle's per-row / per-column form).
 """
 import numpy as np
 import pytest
@@ -20,8 +23,15 @@ pytestmark = pytest.mark.gpu
 VOCAB = 128256
 
 
+def _sample_views(pack, s, tensors, heads, kv_heads):
+    lo, hi = int(pack.cu_seqlens[s]), int(pack.cu_seqlens[s + 1])
+    q, k, v, d_o = tensors
+    f = wl.to_f64
+    return lo, hi, f(q[lo:hi, heads]), f(k[lo:hi, kv_heads]), f(v[lo:hi, kv_heads]), f(d_o[lo:hi, heads])
+
+
 @pytest.mark.parametrize("workload", [1, 2, 3, 4])
-def test_attention_on_whole_samples_of_the_bench_packs(workload):
+def test_attention_on_the_bench_packs(workload):
     pack = wl.config_pack(workload)
     Hq, Hkv, d = pack.n_q_heads, pack.n_kv_heads, pack.head_dim
     g = Hq // Hkv
@@ -31,31 +41,74 @@ def test_attention_on_whole_samples_of_the_bench_packs(workload):
     qd, kd, vd, dod = q.cuda(), k.cuda(), v.cuda(), d_o.cuda()
     o, lse = B.psa_fwd(plan, qd, kd, vd, status=status)
     dq, dk, dv = B.psa_bwd(plan, dod, qd, kd, vd, o, lse, status=status)
+    fq, fk, fv = B.psa_bwd_f32(plan, dod, qd, kd, vd, o, lse, status=status)
     assert read_status(status) == 0
-    o, lse, dq, dk, dv = (t.cpu() for t in (o, lse, dq, dk, dv))
+    o, lse, dq, dk, dv, fq, fk, fv = (t.cpu() for t in (o, lse, dq, dk, dv, fq, fk, fv))
+    del qd, kd, vd, dod
 
     lens = pack.cu_seqlens[1:] - pack.cu_seqlens[:-1]
     rng = np.random.default_rng(workload)
+
+    # ---- (1) whole samples, one kv-head group each, every element (dense oracle)
     small = [s for s in np.argsort(lens) if lens[s] <= 3000]
     picks = sorted({int(small[0]), int(small[-1]), int(rng.choice(small))})
     for s in picks:
         hk = int(rng.integers(0, Hkv))
-        lo, hi = int(pack.cu_seqlens[s]), int(pack.cu_seqlens[s + 1])
         hs = slice(hk * g, hk * g + g)
+        lo, hi, sq, sk, sv, sdo = _sample_views(pack, s, (q, k, v, d_o), hs, slice(hk, hk + 1))
         P, C, R = (int(x[s]) for x in (pack.prefix_len, pack.chosen_len, pack.rejected_len))
         mask = orc.packed_mask([0, hi - lo], [P], [C], [R])
-        f = wl.to_f64
-        sq, sk, sv, sdo = f(q[lo:hi, hs]), f(k[lo:hi, hk:hk + 1]), f(v[lo:hi, hk:hk + 1]), f(d_o[lo:hi, hs])
         ro, rl = orc.attention_fwd(sq, sk, sv, mask)
         rdq, rdk, rdv = orc.attention_bwd(sq, sk, sv, sdo, mask)
         eo, el = max_abs(o[lo:hi, hs], ro), max_abs(lse[hs, lo:hi], rl)
         assert eo <= TOL_O and el <= TOL_LSE, (workload, s, eo, el)
-        for name, got, ref in (("dq", dq[lo:hi, hs], rdq), ("dk", dk[lo:hi, hk:hk + 1], rdk), ("dv", dv[lo:hi, hk:hk + 1], rdv)):
+        for name, got, got32, ref in (("dq", dq[lo:hi, hs], fq[lo:hi, hs], rdq),
+                                      ("dk", dk[lo:hi, hk:hk + 1], fk[lo:hi, hk:hk + 1], rdk),
+                                      ("dv", dv[lo:hi, hk:hk + 1], fv[lo:hi, hk:hk + 1], rdv)):
             raw, raw_small, excess = grad_errors(got, ref)
             assert raw_small <= TOL_O and excess <= TOL_O, (workload, s, name, raw, raw_small, excess)
-    # properties that hold at any size: finite everywhere, lse >= the row's own score
+            raw32 = max_abs(got32, ref)          # fp32 outputs: the gate as stated, raw, on every element
+            print("workload %d sample %d %s: raw max abs error bf16 out %.4f, fp32 out %.4f" % (workload, s, name, raw, raw32))
+            assert raw32 <= TOL_O, (workload, s, name, raw32)
+
+    # ---- (2) sampled over the WHOLE pack and ALL heads: forward rows (random rows of every sample and
+    # every boundary row), and on the longest sample gradients of sampled rows (dq) and of key positions
+    # in the tails of the two responses (dk, dv), where the oracle needs only the rows that see them.
+    all_q, all_kv = slice(0, Hq), slice(0, Hkv)
+    longest = int(np.argmax(lens))
+    for s in range(pack.n_samples):
+        lo, hi, sq, sk, sv, sdo = _sample_views(pack, s, (q, k, v, d_o), all_q, all_kv)
+        L = hi - lo
+        P, C, R = (int(x[s]) for x in (pack.prefix_len, pack.chosen_len, pack.rejected_len))
+        edge = [0, 1, 127, 128, P - 1, P, P + C - 1, P + C, L - 1, (L - 1) // 128 * 128, (L - 1) // 128 * 128 - 1]
+        rows = np.unique(np.clip(np.concatenate([edge, rng.integers(0, L, 14 if s != longest else 40)]), 0, L - 1))
+        mask = orc.packed_mask([0, L], [P], [C], [R])
+        cols = np.zeros(0, dtype=np.int64)
+        need = rows
+        if s == longest:
+            tail = lambda a, b: np.unique(np.clip(np.concatenate([[b - 1, max(a, b - 64)], rng.integers(max(a, b - 64), max(b, a + 1), 6)]), a, max(a, b - 1)))
+            cols = np.unique(np.concatenate([tail(P, P + C) if C else [], tail(P + C, L) if R else []]).astype(np.int64))
+            need = np.unique(np.concatenate([rows, np.nonzero(mask[:, cols].any(axis=1))[0]]))
+        ro, rl = orc.attention_rows(sq, sk, sv, mask[need], need)
+        at = np.searchsorted(need, rows)
+        eo, el = max_abs(o[lo:hi][rows], ro[at]), max_abs(lse[:, lo:hi][:, rows], rl[:, at])
+        assert eo <= TOL_O and el <= TOL_LSE, (workload, s, "sampled rows", eo, el)
+        if s != longest:
+            continue
+        full_o = np.zeros((L, Hq, d)); full_l = np.zeros((Hq, L))
+        full_o[need], full_l[:, need] = ro, rl
+        rdq, rdk, rdv = orc.attention_bwd_sampled(sq, sk, sv, sdo, full_o, full_l, mask, rows, cols)
+        for name, got, got32, ref in (("dq", dq[lo:hi][rows], fq[lo:hi][rows], rdq), ("dk", dk[lo:hi][cols], fk[lo:hi][cols], rdk),
+                                      ("dv", dv[lo:hi][cols], fv[lo:hi][cols], rdv)):
+            raw, raw_small, excess = grad_errors(got, ref)
+            raw32 = max_abs(got32, ref)
+            print("workload %d longest sample (%d tokens) %s, all heads, sampled: raw bf16 out %.4f, fp32 out %.4f"
+                  % (workload, L, name, raw, raw32))
+            assert raw_small <= TOL_O and excess <= TOL_O and raw32 <= TOL_O, (workload, name, raw, raw_small, excess, raw32)
+
+    # ---- (3) properties that hold at any size: finite everywhere, lse >= the row's own score
     assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
-    assert all(torch.isfinite(t.float()).all() for t in (dq, dk, dv))
+    assert all(torch.isfinite(t.float()).all() for t in (dq, dk, dv, fq, fk, fv))
     own = (q.float() * k.float().repeat_interleave(g, dim=1)).sum(-1).t() * d ** -0.5     # [Hq, T]
     assert (lse + 1e-3 >= own).all()
 

@@ -99,3 +99,29 @@ def test_single_row_of_any_width(vocab, dtype):
     grad = B.dpo_logp_bwd(x.cuda(), tok.cuda(), _dev(seg), coef)
     ref = orc.dpo_logp_grad(wl.to_f64(x), tok.numpy(), seg, [0.75])
     assert np.abs(grad.cpu().double().numpy() - ref).max() <= (2e-6 if dtype == torch.float32 else 2.0 ** -8)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_rows_that_begin_with_a_block_of_minus_infinity(dtype):
+    """Banned or padded vocabulary entries are -inf.  A thread whose first chunk of the row is all
+    -inf must carry "nothing yet", not a NaN, into the rest of the row; the gradient sweep too."""
+    n_rows, vocab = 6, 4096
+    x, tok = wl.logits_and_tokens(n_rows, vocab, 21, 2.0, dtype)
+    x[0, :1024] = -float("inf")            # every thread's first chunk (and more)
+    x[1, :32] = -float("inf")              # exactly one thread's first chunk
+    x[2, 100:2100] = -float("inf")         # a block in the middle
+    x[3, vocab - 700:] = -float("inf")     # the tail
+    x[4, ::2] = -float("inf")              # every other entry
+    tok = tok.clone()
+    tok[0], tok[1], tok[2], tok[3], tok[4] = 2000, 40, 50, 7, 1
+    seg = np.arange(n_rows, dtype=np.int32)
+    out = B.dpo_logp(x.cuda(), tok.cuda(), _dev(seg), n_rows)
+    want = orc.dpo_logp(wl.to_f64(x), tok.numpy(), seg, n_rows)
+    got = out.cpu().double().numpy()
+    assert np.isfinite(got).all()
+    assert (np.abs(got - want) / np.abs(want)).max() <= TOL_LOGP
+    coef = torch.linspace(0.1, 0.6, n_rows, dtype=torch.float32).cuda()
+    grad = B.dpo_logp_bwd(x.cuda(), tok.cuda(), _dev(seg), coef).cpu().double().numpy()
+    ref = orc.dpo_logp_grad(wl.to_f64(x), tok.numpy(), seg, coef.cpu().double().numpy())
+    assert np.isfinite(grad).all()
+    assert np.abs(grad - ref).max() <= (2e-6 if dtype == torch.float32 else 2.0 ** -8)

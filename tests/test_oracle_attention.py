@@ -181,3 +181,22 @@ def test_sampled_gradient_equals_the_dense_gradient_on_its_rows_and_columns():
     sq, sk, sv = orc.attention_bwd_sampled(q, k, v, d_o, o2, lse2, mask, rows, cols)
     assert np.abs(sq - dq[rows]).max() < 1e-13
     assert np.abs(sk - dk[cols]).max() < 1e-13 and np.abs(sv - dv[cols]).max() < 1e-13
+
+
+def test_sampled_backward_needs_the_forward_only_on_the_rows_that_see_the_sampled_keys():
+    """The full-size GPU tests call attention_bwd_sampled with o and lse filled in only on the
+    sampled query rows and on the rows that see a sampled key (zeros elsewhere): the result must
+    be the dense gradient at those rows and key positions."""
+    pack = wl.pack_from_lengths("s", [(37, 21, 30)], 4, 2, 16)
+    q, k, v, d_o = (wl.to_f64(t) for t in wl.attention_inputs(pack, 12))
+    mask = orc.packed_mask(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len)
+    dq, dk, dv = orc.attention_bwd(q, k, v, d_o, mask)
+    rows = np.array([0, 5, 36, 37, 57, 58, 87])
+    cols = np.array([50, 57, 80, 87])                      # tails of the chosen and of the rejected response
+    need = np.unique(np.concatenate([rows, np.nonzero(mask[:, cols].any(axis=1))[0]]))
+    assert len(need) < pack.total_tokens - 20              # far from all rows
+    o, lse = np.zeros_like(q), np.zeros((4, pack.total_tokens))
+    o[need], lse[:, need] = orc.attention_rows(q, k, v, mask[need], need)
+    sdq, sdk, sdv = orc.attention_bwd_sampled(q, k, v, d_o, o, lse, mask, rows, cols)
+    assert np.allclose(sdq, dq[rows], atol=1e-12)
+    assert np.allclose(sdk, dk[cols], atol=1e-12) and np.allclose(sdv, dv[cols], atol=1e-12)

@@ -4,10 +4,12 @@ Some callers cannot give psa_bwd a workspace: all device memory may already belo
 the framework's allocator, or the call sits in a loop that must not hit the device-wide
 synchronisation of cudaMalloc / cudaFree.  For them the library keeps a fixed 32 MiB
 scratch array of its own.  This test calls that entry point through the C ABI twice in
-a row and checks both results against the ordinary psa_bwd on the same inputs; the
-second call also proves that what the first one left in the shared array does no harm.
-The file sorts last so that a run stopping at the first failure has already run every
-other test.
+a row and checks both results against the ordinary psa_bwd on the same inputs and against
+the fp64 oracle; the second call also proves that what the first one left in the shared
+array does no harm.  It also checks the claim in the name: across a call (after a first,
+warm-up call, which looks the array's address up) the device's free memory and the
+framework allocator's counters do not move.  The file sorts last so that a run stopping at
+the first failure has already run every other test.
 """
 import numpy as np
 import pytest
@@ -16,7 +18,7 @@ import torch
 from paper_2410_20305_b200 import binding as B
 from paper_2410_20305_b200 import workloads as wl
 
-from gpu_util import TOL_O, device_plan, half_ulp_bf16, read_status
+from gpu_util import TOL_O, device_plan, grad_errors, half_ulp_bf16, oracle_bwd, read_status
 
 pytestmark = pytest.mark.gpu
 
@@ -46,6 +48,29 @@ def test_static_scratch_matches_workspace_entry_point_twice(pack_id):
         for name, a, b in zip(("dq", "dk", "dv"), got, want):
             ok, worst = _close(a, b)
             assert ok, (pack_id, call, name, worst)
+        # and against the oracle, with the gate of the bf16-output gradient tests
+        cpu = wl.attention_inputs(pack, 20 + call)
+        for name, a, ref in zip(("dq", "dk", "dv"), got, oracle_bwd(pack, *cpu)):
+            raw, raw_small, excess = grad_errors(a, ref)
+            assert raw_small <= TOL_O and excess <= TOL_O, (pack_id, call, name, raw, raw_small, excess)
+
+
+def test_the_call_allocates_no_device_memory():
+    pack = wl.config_pack(0)
+    plan = device_plan(pack)
+    q, k, v, d_o = (t.cuda() for t in wl.attention_inputs(pack, 31))
+    o, lse = B.psa_fwd(plan, q, k, v)
+    got = (torch.empty_like(q), torch.empty_like(k), torch.empty_like(v))
+    B.psa_bwd_static_scratch(plan, d_o, q, k, v, o, lse, *got)       # first call on the device: address look-up
+    torch.cuda.synchronize()
+    keys = ("allocation.all.allocated", "segment.all.allocated", "reserved_bytes.all.current", "num_alloc_retries")
+    stats0 = {key: torch.cuda.memory_stats().get(key, 0) for key in keys}
+    free0 = torch.cuda.mem_get_info()[0]
+    for _ in range(3):
+        B.psa_bwd_static_scratch(plan, d_o, q, k, v, o, lse, *got)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0, "device free memory changed across the calls"
+    assert {key: torch.cuda.memory_stats().get(key, 0) for key in keys} == stats0
 
 
 def test_plans_beyond_the_static_scratch_are_rejected():
