@@ -6,7 +6,10 @@ host, psa_fwd, psa_bwd, and dpo_logp over the pack's logits.  The headline metri
 is the useful TFLOP/s of attention forward + backward (14*d*Hq*U flops, U = the
 unmasked (q, kv) pairs per head) over the time of those two calls, measured with
 CUDA events inside the timed steps; packed tokens/s over the whole step and the
-gather's GB/s are reported beside it.
+gather's GB/s are reported beside it.  The default workload is the largest
+single-GPU configuration (multi-turn, a 32768-token pack, with the gather over bf16
+logits of vocabulary 128256); the other three configurations are measured in the
+same process and reported in the line's `workloads` object.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..4] [--impl reference]
 
@@ -16,7 +19,9 @@ path has no exchange step, so there is no collective on the data path.
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
+import math
 import os
 import subprocess
 import sys
@@ -33,10 +38,14 @@ UNIT = "TFLOP/s"
 VOCAB = 128256            # logits width of the gather leg (bf16)
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (read + write) of one psa_bwd_kernel launch, from the ncu capture summarised in
-# profiles/psa_bwd_kernel_llama3-8b.md (workload 1); other workloads have no capture.
+TARGET_FRAC_OF_BF16_PEAK = 0.5      # attention fwd+bwd, useful flops
+TARGET_FRAC_OF_HBM = 0.7            # the gather
+MIN_TIMED_SECONDS = 0.5             # the timed region runs at least this long (inner repeats of the step)
 N_E2E = int(os.environ.get("PSA_BENCH_E2E_STREAMS", "3"))   # arenas / streams of the end-to-end leg
-NCU_BWD_TRAFFIC_BYTES = {1: 1454.7e6}
+ORACLE_SAMPLE_PAIRS = 6.0e6         # useful pairs per head of the oracle's timed sample (about 1.5 s per pass)
+NCU_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+# sources whose text decides the DRAM traffic of the backward's main kernel (kernel, waits, launch order)
+TRAFFIC_SOURCES = ("psa_bwd.cu", "psa_device.cuh", "psa_plan.cpp")
 
 
 def measured_peaks():
@@ -48,6 +57,29 @@ def measured_peaks():
         return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
                 "bf16_tflops_sustained": d.get("bf16_tflops_sustained"), "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def traffic_source_digest():
+    """Digest of the sources that decide the backward kernel's DRAM traffic; an ncu figure taken
+    from another version of them is stale."""
+    h = hashlib.sha256()
+    for name in TRAFFIC_SOURCES:
+        with open(os.path.join(ROOT, "paper_2410_20305_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(kernel, workload_name):
+    """DRAM bytes (read + write) of one launch of `kernel` on `workload_name`, from the tracked
+    summary of an ncu capture (written by paper_2410_20305_b200/ncu_summary.py); None when there
+    is no capture of this workload or it was taken from other kernel sources."""
+    try:
+        rec = json.load(open(NCU_TRAFFIC_FILE))[kernel][workload_name]
+    except (OSError, KeyError, ValueError):
+        return None, "no capture of this kernel on this workload"
+    if rec.get("source_digest") != traffic_source_digest():
+        return None, "stale: captured from other kernel sources (%s)" % rec.get("source_digest")
+    return float(rec["dram_bytes"]), rec.get("command")
 
 
 class ClockSampler:
@@ -124,9 +156,7 @@ class ClockSampler:
         if self.source == "nvml":
             reasons = [n for n in self.NAMES if self.mask & self.BITS[n]]
             return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_min_mhz": min(self.sm) if self.sm else None,
-                    "sm_max_mhz": self.max_sm, "reasons": reasons, "samples": len(self.sm), "source": "nvml, every 2 ms",
-                    "note": "NVML's reading; inside the attention kernels ncu's sm__cycles_elapsed.avg.per_second is "
-                            "1.59-1.68 GHz (see profiles/), with no clock-event reason raised"}
+                    "sm_max_mhz": self.max_sm, "reasons": reasons, "samples": len(self.sm), "source": "nvml, every 2 ms"}
         sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
         mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
         reasons = [n for i, n in enumerate(self.NAMES) if any(len(r) >= 6 and r[2 + i] == "Active" for r in self.rows)]
@@ -150,17 +180,29 @@ def whole_job_tflops(flops_per_replica, world, ms):
     return world * flops_per_replica / ms / 1e9
 
 
-def oracle_sample(pack, steps, warmup, target="bench"):
-    """Times the fp64 oracle, as it stands, on a bounded sample of the workload: whole
-    samples of the pack (attention is independent per sample, which the oracle's own tests
-    pin) for one kv group of 4 query heads.  The baseline leg takes every sample of the
-    pack (1/8 of the workload's heads), the reference arm only the shortest sample because
-    it runs many steps.  Returns (useful TFLOP/s, description, cores, seconds per step)."""
+def oracle_sample_set(pack):
+    """The bounded sample of the workload that both oracle legs time: whole samples of the pack
+    (attention is independent per sample, which the oracle's own tests pin), taken at every second
+    rank of the samples sorted by length so that the length mix is the pack's, until their useful
+    pairs reach ORACLE_SAMPLE_PAIRS; one kv-head group (4 query heads, 1 kv head)."""
+    from oracle import psa_oracle as orc
+    order = np.argsort(pack.cu_seqlens[1:] - pack.cu_seqlens[:-1], kind="stable")
+    chosen, pairs = [], 0
+    for s in [int(x) for x in order[0::2]]:
+        chosen.append(s)
+        pairs += orc.useful_pairs([pack.prefix_len[s]], [pack.chosen_len[s]], [pack.rejected_len[s]])
+        if pairs >= ORACLE_SAMPLE_PAIRS:
+            break
+    return chosen
+
+
+def oracle_sample(pack, steps, warmup):
+    """Times the fp64 oracle, as it stands, on oracle_sample_set(pack): forward and backward, dense
+    mask, numpy.  Returns (useful TFLOP/s, description, cores, seconds per step)."""
     import torch
     from oracle import psa_oracle as orc
     from paper_2410_20305_b200 import workloads as wl
-    order = np.argsort(pack.cu_seqlens[1:] - pack.cu_seqlens[:-1])
-    chosen = [int(x) for x in (order if target == "bench" else order[:1])]
+    chosen = oracle_sample_set(pack)
     subs, flops = [], 0.0
     for s in chosen:
         P, C, R = int(pack.prefix_len[s]), int(pack.chosen_len[s]), int(pack.rejected_len[s])
@@ -178,16 +220,19 @@ def oracle_sample(pack, steps, warmup, target="bench"):
         if i >= warmup:
             times.append(time.perf_counter() - t0)
     sec = float(np.mean(times))
-    desc = "%d sample(s) of the pack (%d tokens), 4 query heads / 1 kv head, fwd+bwd, dense fp64 numpy" % (
-        len(chosen), int(sum(pack.cu_seqlens[s + 1] - pack.cu_seqlens[s] for s in chosen)))
+    desc = "%d of the pack's %d samples (%d of %d tokens, every second one by length), 4 query heads / 1 kv head, " \
+           "fwd+bwd, dense fp64 numpy" % (len(chosen), pack.n_samples,
+                                          int(sum(pack.cu_seqlens[s + 1] - pack.cu_seqlens[s] for s in chosen)),
+                                          pack.total_tokens)
     return flops / sec / 1e12, desc, torch.get_num_threads(), sec
 
 
 def run_reference(args, pack, rank):
-    """The reference arm: the CPU oracle on the machine's host cores, rank 0 only."""
+    """The reference arm: the CPU oracle on the machine's host cores, rank 0 only, on the same sample
+    as the cpu_baseline leg of the main arm."""
     if rank != 0:
         return
-    val, desc, cores, sec = oracle_sample(pack, args.steps, args.warmup, target="reference")
+    val, desc, cores, sec = oracle_sample(pack, args.steps, args.warmup)
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -197,18 +242,76 @@ def run_reference(args, pack, rank):
     print(json.dumps(line))
 
 
+def attention_record(index, dev, peaks, iters=30, warm=5):
+    """Attention fwd+bwd of workload `index` on the shared layout and, with the same kernels, on the
+    unshared paired layout: ms, useful TFLOP/s, fractions of the bf16 peaks, tokens/s, speed-up."""
+    import torch
+    from paper_2410_20305_b200 import binding as B
+    from paper_2410_20305_b200 import workloads as wl
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(pk, seed):
+        Hq, Hkv, d = pk.n_q_heads, pk.n_kv_heads, pk.head_dim
+        q, k, v, d_o = (t.to(dev) for t in wl.attention_inputs(pk, seed))
+        plan = B.psa_plan(pk.cu_seqlens, pk.prefix_len, pk.chosen_len, pk.rejected_len, Hq, Hkv, d)
+        o, lse = B.psa_fwd(plan, q, k, v)
+        ws = torch.empty(plan.bwd_workspace_bytes, dtype=torch.uint8, device=dev)
+        dq, dk, dv = B.psa_bwd(plan, d_o, q, k, v, o, lse, workspace=ws)
+        for _ in range(warm):
+            B.psa_fwd(plan, q, k, v, o=o, lse=lse)
+            B.psa_bwd(plan, d_o, q, k, v, o, lse, dq=dq, dk=dk, dv=dv, workspace=ws)
+        torch.cuda.synchronize()
+        a, m, b = ev(), ev(), ev()
+        fwd_ms = 0.0
+        a.record()
+        for _ in range(iters):
+            B.psa_fwd(plan, q, k, v, o=o, lse=lse)
+            B.psa_bwd(plan, d_o, q, k, v, o, lse, dq=dq, dk=dk, dv=dv, workspace=ws)
+        b.record()
+        torch.cuda.synchronize()
+        total = a.elapsed_time(b) / iters
+        a.record()
+        for _ in range(iters):
+            B.psa_fwd(plan, q, k, v, o=o, lse=lse)
+        m.record()
+        torch.cuda.synchronize()
+        fwd_ms = a.elapsed_time(m) / iters
+        return total, fwd_ms, plan.useful_pairs, plan.live_tiles
+
+    pack = wl.config_pack(index)
+    Hq, Hkv, d, T = pack.n_q_heads, pack.n_kv_heads, pack.head_dim, pack.total_tokens
+    ms, fwd_ms, U, live = timed(pack, 2000 + index)
+    pp = pack.paired()
+    p_ms, _, pU, _ = timed(pp, 2100 + index)
+    torch.cuda.empty_cache()
+    tflops = 14.0 * d * Hq * U / ms / 1e9
+    min_bytes = T * (6 * Hq + 6 * Hkv) * d * 2
+    return {"workload": pack.name, "total_tokens": T, "n_samples": pack.n_samples, "useful_pairs_per_head": U,
+            "live_tiles": live, "attention_fwd_bwd_ms": ms, "fwd_ms_back_to_back": fwd_ms, "useful_tflops": tflops,
+            "pct_of_bf16_peak": {"measured": tflops / peaks["bf16_tflops"], "nominal": tflops / NOMINAL_BF16_TFLOPS},
+            "attention_tokens_per_s": T / (ms * 1e-3),
+            "attention_min_hbm_frac": {"measured": min_bytes / ms / 1e6 / peaks["hbm_gbs"],
+                                       "nominal": min_bytes / ms / 1e6 / NOMINAL_HBM_GBS},
+            "paired_layout": {"tokens": pp.total_tokens, "fwd_bwd_ms": p_ms, "speedup_shared_over_paired": p_ms / ms,
+                              "ideal_pair_ratio": pU / U, "token_ratio": pp.total_tokens / T},
+            "timing": "%d iterations after %d warm-up, CUDA events, inputs larger than L2" % (iters, warm)}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="psa", choices=["psa", "reference"])
-    ap.add_argument("--workload", type=int, default=1, help="1 llama3-8b, 2 long-prompt, 3 multi-turn, 4 short-many")
+    ap.add_argument("--workload", type=int, default=3, choices=[1, 2, 3, 4],
+                    help="1 llama3-8b, 2 long-prompt, 3 multi-turn (default: the largest single-GPU configuration), 4 short-many")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-layer", action="store_true")
     ap.add_argument("--no-paired", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the records of the other three configurations")
     ap.add_argument("--no-logp", action="store_true", help="attention only (small footprint, for ncu captures)")
+    ap.add_argument("--no-inner-repeats", action="store_true", help="time exactly --steps passes (for ncu captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -224,6 +327,7 @@ def main():
     import torch.distributed as dist
     import paper_2410_20305_b200 as psa
     from paper_2410_20305_b200 import binding as B
+    from paper_2410_20305_b200.layer import AttentionLayer
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
@@ -231,6 +335,7 @@ def main():
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    peaks = measured_peaks()
 
     T, Hq, Hkv, d = pack.total_tokens, pack.n_q_heads, pack.n_kv_heads, pack.head_dim
     q, k, v, d_o = (t.to(dev) for t in wl.attention_inputs(pack, 2000 + args.workload, std=1.0))
@@ -257,20 +362,21 @@ def main():
     flops_fwd, flops_bwd = 4.0 * d * Hq * U, 10.0 * d * Hq * U
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    n_total = args.warmup + args.steps
-    e_att0, e_att1, e_lp1 = [ev() for _ in range(n_total)], [ev() for _ in range(n_total)], [ev() for _ in range(n_total)]
     k_fwd, k_bwd, k_lp = (ev(), ev()), (ev(), ev()), (ev(), ev())
     kernel_ms = {"fwd": [], "bwd": [], "logp": []}
 
-    def step(i, timed):
+    def step(e0=None, e1=None, e2=None):
         plan = B.psa_plan(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len, Hq, Hkv, d)
-        e_att0[i].record()
+        if e0 is not None:
+            e0.record()
         B.psa_fwd(plan, q, k, v, o=o, lse=lse, status=status)
         B.psa_bwd(plan, d_o, q, k, v, o, lse, dq=dq, dk=dk, dv=dv, workspace=ws, status=status)
-        e_att1[i].record()
+        if e1 is not None:
+            e1.record()
         if not args.no_logp:
             B.dpo_logp(logits, targets, seg_d, n_seg, fr, ft, fs, out=logp, status=status)
-        e_lp1[i].record()
+        if e2 is not None:
+            e2.record()
         return plan
 
     def sync_all():
@@ -285,15 +391,27 @@ def main():
         B.psa_plan(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len, Hq, Hkv, d).close()
     plan_host_ms = (time.perf_counter() - t0) * 1e3 / 20
 
+    # Warm-up; the last warm-up steps also give the step's duration, from which the number of inner
+    # repeats follows: the timed region is to last at least MIN_TIMED_SECONDS whatever --steps is.
+    for i in range(args.warmup):
+        step()
+    sync_all()
+    a, b = ev(), ev()
+    a.record()
+    for _ in range(3):
+        step()
+    b.record()
+    sync_all()
+    est_ms = a.elapsed_time(b) / 3
+    inner = 1 if args.no_inner_repeats else max(1, int(math.ceil(MIN_TIMED_SECONDS * 1e3 / (args.steps * est_ms))))
+    n_pass = args.steps * inner
+
     # Per-kernel events (the library records them right around each main kernel) are read one
     # step at a time in a separate short pass so that the timed region below stays free of syncs.
-    for i in range(args.warmup):
-        step(i, False)
-    sync_all()
     for name, which, pair in (("fwd", 0, k_fwd), ("bwd", 1, k_bwd), ("logp", 2, k_lp)):
         B.psa_profile_events(which, *pair)
     for i in range(min(args.steps, 10)):
-        step(0, False)
+        step()
         torch.cuda.synchronize()
         for name, pair in (("fwd", k_fwd), ("bwd", k_bwd), ("logp", k_lp)):
             if name == "logp" and args.no_logp:
@@ -303,18 +421,20 @@ def main():
     for which in range(3):
         B.psa_profile_events(which)
 
+    e_att0, e_att1, e_lp1 = [ev() for _ in range(n_pass)], [ev() for _ in range(n_pass)], [ev() for _ in range(n_pass)]
     sync_all()
     t_start, t_stop = ev(), ev()
     with ClockSampler(local_rank) as clocks:
         t_start.record()
-        for i in range(args.warmup, n_total):
-            step(i, True)
+        for i in range(n_pass):
+            step(e_att0[i], e_att1[i], e_lp1[i])
         t_stop.record()
         sync_all()
-    step_ms = t_start.elapsed_time(t_stop) / args.steps
-    att_all = [e_att0[i].elapsed_time(e_att1[i]) for i in range(args.warmup, n_total)]
+    timed_ms = t_start.elapsed_time(t_stop)
+    step_ms = timed_ms / n_pass
+    att_all = [e_att0[i].elapsed_time(e_att1[i]) for i in range(n_pass)]
     att_ms = float(np.mean(att_all))
-    lp_ms = float(np.mean([e_att1[i].elapsed_time(e_lp1[i]) for i in range(args.warmup, n_total)]))
+    lp_ms = float(np.mean([e_att1[i].elapsed_time(e_lp1[i]) for i in range(n_pass)]))
     if int(status.item()) != 0:
         raise SystemExit("device status word is %d: results invalid" % int(status.item()))
 
@@ -356,6 +476,8 @@ def main():
         ar_ms = a.elapsed_time(b) / 5
         ar_bytes = T * (VOCAB * 2 + 8)
         all_rows = {"rows": T, "ms": ar_ms, "gbs": ar_bytes / ar_ms / 1e6, "algorithmic_bytes": ar_bytes}
+    del logits
+    torch.cuda.empty_cache()
 
     # ---- the same kernels on the unshared paired layout (2n causal sequences)
     paired = None
@@ -368,57 +490,56 @@ def main():
         pdq, pdk, pdv = B.psa_bwd(pplan, pdo, pq, pk, pv, po, plse, workspace=pws)
         torch.cuda.synchronize()
         a, b = ev(), ev()
+        n_p = max(args.steps, 20)
         a.record()
-        for _ in range(args.steps):
+        for _ in range(n_p):
             B.psa_fwd(pplan, pq, pk, pv, o=po, lse=plse)
             B.psa_bwd(pplan, pdo, pq, pk, pv, po, plse, dq=pdq, dk=pdk, dv=pdv, workspace=pws)
         b.record()
         torch.cuda.synchronize()
-        p_ms = a.elapsed_time(b) / args.steps
+        p_ms = a.elapsed_time(b) / n_p
         paired = {"tokens": pp.total_tokens, "fwd_bwd_ms": p_ms, "speedup_shared_over_paired": p_ms / att_ms,
                   "ideal_pair_ratio": pplan.useful_pairs / U, "token_ratio": pp.total_tokens / T}
         del pq, pk, pv, pdo, po, plse, pws, pdq, pdk, pdv
+        torch.cuda.empty_cache()
+
+    # ---- the other three configurations, measured here and now with the same build
+    others = None
+    if not args.no_workloads and rank == 0:
+        others = {}
+        for w in (1, 2, 3, 4):
+            if w != args.workload:
+                rec = attention_record(w, dev, peaks)
+                others[rec["workload"]] = rec
 
     # ---- attention-layer level (a "next" row): QKV and output projections (library GEMMs through
     # torch.matmul), rotary embedding on the shared layout's position ids, psa_fwd / psa_bwd, and the
-    # projections' backward; the same on the paired layout.
+    # projections' backward (paper_2410_20305_b200/layer.py); the same on the paired layout.
     layer = None
     if not args.no_layer and rank == 0:
         def layer_ms(pk_, seed):
-            Tl = pk_.total_tokens
-            hid = Hq * d
+            Tl, hid = pk_.total_tokens, Hq * d
             g = torch.Generator(device=dev); g.manual_seed(seed)
             rn = lambda *shape: (torch.randn(*shape, generator=g, device=dev) * 0.02).to(torch.bfloat16)
             x = (torch.randn(Tl, hid, generator=g, device=dev)).to(torch.bfloat16)
             dout = (torch.randn(Tl, hid, generator=g, device=dev)).to(torch.bfloat16)
             wq, wk, wv, wo = rn(hid, Hq * d), rn(hid, Hkv * d), rn(hid, Hkv * d), rn(Hq * d, hid)
-            pos = torch.as_tensor(B.psa_position_ids(pk_.cu_seqlens, pk_.prefix_len, pk_.chosen_len, pk_.rejected_len)).to(dev)
-            neg = -pos
-            lplan = B.psa_plan(pk_.cu_seqlens, pk_.prefix_len, pk_.chosen_len, pk_.rejected_len, Hq, Hkv, d)
-            lws = torch.empty(lplan.bwd_workspace_bytes, dtype=torch.uint8, device=dev)
+            lay = AttentionLayer((pk_.cu_seqlens, pk_.prefix_len, pk_.chosen_len, pk_.rejected_len), Hq, Hkv, d, dev)
 
             def run():
-                q_ = (x @ wq).view(Tl, Hq, d); k_ = (x @ wk).view(Tl, Hkv, d); v_ = (x @ wv).view(Tl, Hkv, d)
-                B.psa_rope(q_, pos, out=q_); B.psa_rope(k_, pos, out=k_)
-                o_, lse_ = B.psa_fwd(lplan, q_, k_, v_)
-                out = o_.view(Tl, hid) @ wo                                   # noqa: F841  (the layer's output)
-                do_ = (dout @ wo.t()).view(Tl, Hq, d)
-                dwo = o_.view(Tl, hid).t() @ dout                             # noqa: F841
-                dq_, dk_, dv_ = B.psa_bwd(lplan, do_, q_, k_, v_, o_, lse_, workspace=lws)
-                B.psa_rope(dq_, neg, out=dq_); B.psa_rope(dk_, neg, out=dk_)   # gradient of a rotation: the inverse rotation
-                dq2, dk2, dv2 = dq_.view(Tl, -1), dk_.view(Tl, -1), dv_.view(Tl, -1)
-                dx = dq2 @ wq.t() + dk2 @ wk.t() + dv2 @ wv.t()               # noqa: F841
-                dwq, dwk, dwv = x.t() @ dq2, x.t() @ dk2, x.t() @ dv2         # noqa: F841
+                out, saved = lay.forward(x, wq, wk, wv, wo)
+                lay.backward(x, wq, wk, wv, wo, saved, dout)
             for _ in range(3):
                 run()
             torch.cuda.synchronize()
             a, b = ev(), ev()
+            n_l = max(10, min(args.steps, 30))
             a.record()
-            for _ in range(args.steps):
+            for _ in range(n_l):
                 run()
             b.record()
             torch.cuda.synchronize()
-            return a.elapsed_time(b) / args.steps
+            return a.elapsed_time(b) / n_l
         l_shared = layer_ms(pack, 2200 + args.workload)
         l_paired = layer_ms(pack.paired(), 2300 + args.workload)
         layer = {"hidden": Hq * d, "shared_fwd_bwd_ms": l_shared, "paired_fwd_bwd_ms": l_paired,
@@ -427,18 +548,21 @@ def main():
         torch.cuda.empty_cache()
 
     # ---- packing (a "next" row, host only): first-fit-decreasing over 2000 units of the workload's
-    # length distribution, shared units (P + C + R) against paired units (2P + C + R)
+    # length distribution, shared units (P + C + R) against paired units (2P + C + R), laid out for psa_plan
     packing = None
     if rank == 0:
         lens, cap = wl.sample_lengths(args.workload, 2000, 3000 + args.workload)
-        shared = [p + c + r for p, c, r in lens]
-        paired_u = [min(2 * p + c + r, cap) for p, c, r in lens]   # (a unit longer than a pack would be truncated)
+        lens = [(p, c, r) for p, c, r in lens if 2 * p + c + r <= cap]   # (a paired unit longer than a pack would be truncated)
+        P_, C_, R_ = ([x[i] for x in lens] for i in range(3))
         t0 = time.perf_counter()
-        _, nb_s = B.psa_pack_ffd(shared, cap)
-        _, nb_p = B.psa_pack_ffd(paired_u, cap)
-        packing = {"units": len(lens), "pack_len": cap, "packs_shared": nb_s, "packs_paired": nb_p,
-                   "packs_ratio_paired_over_shared": nb_p / nb_s, "fill_shared": sum(shared) / (nb_s * cap),
-                   "fill_paired": sum(paired_u) / (nb_p * cap), "ms_both": (time.perf_counter() - t0) * 1e3}
+        _, packs_s = B.psa_pack_ffd_emit(P_, C_, R_, cap)
+        _, packs_p = B.psa_pack_ffd_emit(P_, C_, R_, cap, paired=True)
+        ms_both = (time.perf_counter() - t0) * 1e3
+        tok_s = sum(int(pk["cu_seqlens"][-1]) for pk in packs_s)
+        tok_p = sum(int(pk["cu_seqlens"][-1]) for pk in packs_p)
+        packing = {"units": len(lens), "pack_len": cap, "packs_shared": len(packs_s), "packs_paired": len(packs_p),
+                   "packs_ratio_paired_over_shared": len(packs_p) / len(packs_s), "fill_shared": tok_s / (len(packs_s) * cap),
+                   "fill_paired": tok_p / (len(packs_p) * cap), "ms_both": ms_both, "call": "psa_pack_ffd_emit"}
 
     # ---- end to end: psa_step_host on pinned host buffers (copies in, fwd, bwd, copies out per step).
     # A few arenas, each on a stream of its own, so that one step's copies out overlap the next step's copies in
@@ -482,7 +606,8 @@ def main():
         assert (last[2].float() - dq.cpu().float()).abs().max().item() <= 0.0625, "psa_step_host: dq differs"
         e2e = {"value": (flops_fwd + flops_bwd) / e2e_ms / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "call": "psa_step_host, %d arenas on %d streams" % (N_E2E, N_E2E), "steps": n_e2e}
+               "call": "psa_step_host, %d arenas on %d streams" % (N_E2E, N_E2E), "steps": n_e2e,
+               "note": "attention forward + backward through host buffers; the gather is not part of this call"}
         del arenas
 
     # ---- max over ranks (replicas): whole-job value = sum of the replicas' useful flops / slowest time
@@ -493,7 +618,6 @@ def main():
             dist.destroy_process_group()
         return
 
-    peaks = measured_peaks()
     if all_rows:
         all_rows["frac_of_hbm"] = {"measured": all_rows["gbs"] / peaks["hbm_gbs"], "nominal": all_rows["gbs"] / NOMINAL_HBM_GBS}
     value = whole_job_tflops(flops_fwd + flops_bwd, world, att_ms)
@@ -501,6 +625,11 @@ def main():
     bwd_ms, fwd_ms, klp_ms = (float(np.mean(kernel_ms[n])) for n in ("bwd", "fwd", "logp"))
     bwd_tflops = flops_bwd / bwd_ms / 1e9
     logp_bytes = live_rows * VOCAB * 2 + 8 * live_rows + 4 * n_seg
+    clk = clocks.summary()
+    sm_mhz = clk.get("sm_mhz")
+    traffic, traffic_note = ncu_traffic("psa_bwd_kernel", pack.name)
+    frac_meas, frac_nom = value / world / peaks["bf16_tflops"], value / world / NOMINAL_BF16_TFLOPS
+    logp_frac_meas = logp_bytes / klp_ms / 1e6 / peaks["hbm_gbs"] if not args.no_logp else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -508,14 +637,27 @@ def main():
         "config": {"workload": pack.name, "pack_len": pack.pack_len, "total_tokens": T, "n_samples": pack.n_samples,
                    "n_q_heads": Hq, "n_kv_heads": Hkv, "head_dim": d, "useful_pairs_per_head": U,
                    "live_tiles": plan0.live_tiles, "partial_tiles": plan0.partial_tiles, "logits": [T, VOCAB],
-                   "l2": "inputs larger than L2 (q, o, dO, dq are 133 MB each; logits %.1f GB)" % (T * VOCAB * 2 / 1e9),
+                   "l2": "inputs larger than L2 (q, o, dO, dq are %.0f MB each; logits %.1f GB)" % (T * Hq * d * 2 / 1e6, T * VOCAB * 2 / 1e9),
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "inner_repeats": inner,
+        "timed_region": {"passes": n_pass, "ms": timed_ms,
+                         "note": "each of the --steps steps is run inner_repeats times so that the region lasts at least "
+                                 "%.1f s; every figure is per pass" % MIN_TIMED_SECONDS},
         "attention_fwd_bwd_ms": att_ms,
         "attention_fwd_bwd_ms_median_min": [float(np.median(att_all)), float(np.min(att_all))],
+        # duration x clock: what the same work would cost at another SM clock (the part is power-limited under
+        # tensor load; NVML's samples are the only clock reading a program can take without touching any setting)
+        "attention_fwd_bwd_ms_x_sm_mhz": att_ms * sm_mhz if sm_mhz else None,
         "plan_ms_host": plan_host_ms,
         "plan_ms_host_per_layer_of_32": plan_host_ms / 32,   # one plan serves every layer of a step
-        "pct_of_bf16_peak": {"measured": value / world / peaks["bf16_tflops"], "nominal": value / world / NOMINAL_BF16_TFLOPS,
-                             "peak_source": peaks["source"]},
+        "pct_of_bf16_peak": {"measured": frac_meas, "nominal": frac_nom, "peak_source": peaks["source"]},
+        "target": {"attention_fwd_bwd_frac_of_bf16_peak": TARGET_FRAC_OF_BF16_PEAK,
+                   "met_against_measured_peak": bool(frac_meas >= TARGET_FRAC_OF_BF16_PEAK),
+                   "met_against_nominal_peak": bool(frac_nom >= TARGET_FRAC_OF_BF16_PEAK),
+                   "gather_frac_of_hbm": TARGET_FRAC_OF_HBM,
+                   "gather_met_against_measured": None if logp_frac_meas is None else bool(logp_frac_meas >= TARGET_FRAC_OF_HBM),
+                   "gather_met_against_nominal": None if logp_frac_meas is None else
+                   bool(logp_bytes / klp_ms / 1e6 / NOMINAL_HBM_GBS >= TARGET_FRAC_OF_HBM)},
         # the other bound of attention fwd+bwd: six passes over Hq-sized and six over Hkv-sized tensors
         # (the short-many workload sits below the ridge point and is bounded by this one)
         "attention_min_hbm": {"bytes": att_min_bytes, "gbs": att_min_bytes / att_ms / 1e6,
@@ -524,19 +666,24 @@ def main():
         "tokens_per_s": world * T / (step_ms * 1e-3),
         "attention_tokens_per_s": world * T / (att_ms * 1e-3),
         "kernels": {"psa_fwd_ms": fwd_ms, "psa_fwd_tflops": flops_fwd / fwd_ms / 1e9,
+                    "psa_fwd_frac_of_measured_peak": flops_fwd / fwd_ms / 1e9 / peaks["bf16_tflops"],
                     "psa_bwd_main_ms": bwd_ms, "psa_bwd_main_tflops": bwd_tflops,
+                    "psa_bwd_helpers_ms": att_ms - fwd_ms - bwd_ms,
                     "dpo_logp_ms": klp_ms, "dpo_logp_gbs": logp_bytes / klp_ms / 1e6,
                     "dpo_logp_frac_of_hbm": {"measured": logp_bytes / klp_ms / 1e6 / peaks["hbm_gbs"],
                                              "nominal": logp_bytes / klp_ms / 1e6 / NOMINAL_HBM_GBS},
                     "dpo_logp_live_rows": live_rows, "dpo_logp_step_ms": lp_ms},
-        "roofline": {"kernel": "psa_bwd_kernel<128>", "bound": "tensor", "achieved": bwd_tflops,
+        "roofline": {"kernel": "psa_bwd_kernel<%d>" % d, "bound": "tensor", "achieved": bwd_tflops,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": bwd_tflops / peaks["bf16_tflops"],
+                     "scope": "this one kernel (the dominant one), not the attention forward + backward as a whole: "
+                              "that is pct_of_bf16_peak",
                      "peak_kind": "burst bf16 cuBLAS, of " + peaks["source"],
-                     "algorithmic_flops": flops_bwd, "algorithmic_bytes": 40960.0 * T if (Hq, Hkv, d) == (32, 8, 128) else None,
-                     "traffic": NCU_BWD_TRAFFIC_BYTES.get(args.workload)},
-        "clocks": clocks.summary(),
-        "gpu_launches": args.steps * (4 if args.no_logp else 5),
+                     "algorithmic_flops": flops_bwd, "algorithmic_bytes": T * (4 * Hq + 4 * Hkv) * d * 2,
+                     "traffic": traffic, "traffic_source": traffic_note},
+        "clocks": clk,
+        "gpu_launches": n_pass * (4 if args.no_logp else 5),
         "paired_layout": paired,
+        "workloads": others,
         "dpo_logp_all_rows": all_rows,
         "next_rows": loss_bwd,
         "attention_layer": layer,
@@ -548,10 +695,10 @@ def main():
         e2e["ms_per_step"] = e2e_ms_max
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
-        # one untimed and three timed passes over the sample: about 13 s of host work on workload 1
-        val, desc, cores, sec = oracle_sample(pack, 3, 1)
+        # two untimed and eight timed passes over the sample: about 15 s of host work
+        val, desc, cores, sec = oracle_sample(pack, 8, 2)
         line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
-                                "seconds_per_pass": sec, "timed_passes": 3}
+                                "seconds_per_pass": sec, "timed_passes": 8}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
