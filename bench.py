@@ -362,10 +362,13 @@ def main():
     flops_fwd, flops_bwd = 4.0 * d * Hq * U, 10.0 * d * Hq * U
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    k_fwd, k_bwd, k_lp = (ev(), ev()), (ev(), ev()), (ev(), ev())
-    kernel_ms = {"fwd": [], "bwd": [], "logp": []}
+    KERNELS = (("fwd", 0), ("bwd", 1), ("logp", 2), ("bwd_delta_clear", 3), ("bwd_convert", 4))
 
-    def step(e0=None, e1=None, e2=None):
+    def step(e0=None, e1=None, e2=None, kev=None):
+        # kev: this pass's own event pairs, which the library records right around each kernel
+        if kev is not None:
+            for (name, which), pair in zip(KERNELS, kev):
+                B.psa_profile_events(which, pair[0], pair[1], created=True)
         plan = B.psa_plan(pack.cu_seqlens, pack.prefix_len, pack.chosen_len, pack.rejected_len, Hq, Hkv, d)
         if e0 is not None:
             e0.record()
@@ -406,30 +409,27 @@ def main():
     inner = 1 if args.no_inner_repeats else max(1, int(math.ceil(MIN_TIMED_SECONDS * 1e3 / (args.steps * est_ms))))
     n_pass = args.steps * inner
 
-    # Per-kernel events (the library records them right around each main kernel) are read one
-    # step at a time in a separate short pass so that the timed region below stays free of syncs.
-    for name, which, pair in (("fwd", 0, k_fwd), ("bwd", 1, k_bwd), ("logp", 2, k_lp)):
-        B.psa_profile_events(which, *pair)
-    for i in range(min(args.steps, 10)):
-        step()
-        torch.cuda.synchronize()
-        for name, pair in (("fwd", k_fwd), ("bwd", k_bwd), ("logp", k_lp)):
-            if name == "logp" and args.no_logp:
-                kernel_ms[name].append(float("nan"))
-            else:
-                kernel_ms[name].append(pair[0].elapsed_time(pair[1]))
-    for which in range(3):
-        B.psa_profile_events(which)
-
+    # Every pass of the timed region has its own events: around the attention calls, after the
+    # gather, and (recorded by the library itself) right around each kernel.  They are created, i.e.
+    # recorded once, before the region starts; nothing inside the region synchronises.
     e_att0, e_att1, e_lp1 = [ev() for _ in range(n_pass)], [ev() for _ in range(n_pass)], [ev() for _ in range(n_pass)]
+    k_ev = [[(ev(), ev()) for _ in KERNELS] for _ in range(n_pass)]
+    for pairs in k_ev:
+        for a_, b_ in pairs:
+            a_.record(); b_.record()
     sync_all()
     t_start, t_stop = ev(), ev()
     with ClockSampler(local_rank) as clocks:
         t_start.record()
         for i in range(n_pass):
-            step(e_att0[i], e_att1[i], e_lp1[i])
+            step(e_att0[i], e_att1[i], e_lp1[i], k_ev[i])
         t_stop.record()
         sync_all()
+    for _, which in KERNELS:
+        B.psa_profile_events(which)
+    kernel_ms = {name: float(np.mean([k_ev[i][j][0].elapsed_time(k_ev[i][j][1]) for i in range(n_pass)]))
+                 for j, (name, _) in enumerate(KERNELS) if not (name == "logp" and args.no_logp)}
+    kernel_ms.setdefault("logp", float("nan"))
     timed_ms = t_start.elapsed_time(t_stop)
     step_ms = timed_ms / n_pass
     att_all = [e_att0[i].elapsed_time(e_att1[i]) for i in range(n_pass)]
@@ -622,13 +622,19 @@ def main():
         all_rows["frac_of_hbm"] = {"measured": all_rows["gbs"] / peaks["hbm_gbs"], "nominal": all_rows["gbs"] / NOMINAL_HBM_GBS}
     value = whole_job_tflops(flops_fwd + flops_bwd, world, att_ms)
     att_min_bytes = T * (6 * Hq + 6 * Hkv) * d * 2
-    bwd_ms, fwd_ms, klp_ms = (float(np.mean(kernel_ms[n])) for n in ("bwd", "fwd", "logp"))
+    bwd_ms, fwd_ms, klp_ms = kernel_ms["bwd"], kernel_ms["fwd"], kernel_ms["logp"]
+    # A region of half a second or more runs under the power cap at a reduced SM clock: the peak to
+    # read it against is the sustained one (a cuBLAS loop of seconds); a short region against the burst.
+    sustained = timed_ms >= 400.0 and peaks.get("bf16_tflops_sustained")
+    peak_tc = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    peak_kind = ("sustained" if sustained else "burst") + " bf16 cuBLAS, of " + peaks["source"]
     bwd_tflops = flops_bwd / bwd_ms / 1e9
     logp_bytes = live_rows * VOCAB * 2 + 8 * live_rows + 4 * n_seg
     clk = clocks.summary()
     sm_mhz = clk.get("sm_mhz")
     traffic, traffic_note = ncu_traffic("psa_bwd_kernel", pack.name)
     frac_meas, frac_nom = value / world / peaks["bf16_tflops"], value / world / NOMINAL_BF16_TFLOPS
+    frac_sus = value / world / peaks["bf16_tflops_sustained"] if peaks.get("bf16_tflops_sustained") else None
     logp_frac_meas = logp_bytes / klp_ms / 1e6 / peaks["hbm_gbs"] if not args.no_logp else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -650,9 +656,14 @@ def main():
         "attention_fwd_bwd_ms_x_sm_mhz": att_ms * sm_mhz if sm_mhz else None,
         "plan_ms_host": plan_host_ms,
         "plan_ms_host_per_layer_of_32": plan_host_ms / 32,   # one plan serves every layer of a step
-        "pct_of_bf16_peak": {"measured": frac_meas, "nominal": frac_nom, "peak_source": peaks["source"]},
+        "pct_of_bf16_peak": {"measured": frac_meas, "measured_sustained": frac_sus, "nominal": frac_nom,
+                             "peak_source": peaks["source"],
+                             "note": "measured = burst cuBLAS rate (%.1f), measured_sustained = the same GEMM looped for "
+                                     "seconds under the power cap (%s); the timed region here lasts %.2f s"
+                                     % (peaks["bf16_tflops"], peaks.get("bf16_tflops_sustained"), timed_ms * 1e-3)},
         "target": {"attention_fwd_bwd_frac_of_bf16_peak": TARGET_FRAC_OF_BF16_PEAK,
                    "met_against_measured_peak": bool(frac_meas >= TARGET_FRAC_OF_BF16_PEAK),
+                   "met_against_measured_sustained_peak": None if frac_sus is None else bool(frac_sus >= TARGET_FRAC_OF_BF16_PEAK),
                    "met_against_nominal_peak": bool(frac_nom >= TARGET_FRAC_OF_BF16_PEAK),
                    "gather_frac_of_hbm": TARGET_FRAC_OF_HBM,
                    "gather_met_against_measured": None if logp_frac_meas is None else bool(logp_frac_meas >= TARGET_FRAC_OF_HBM),
@@ -668,16 +679,18 @@ def main():
         "kernels": {"psa_fwd_ms": fwd_ms, "psa_fwd_tflops": flops_fwd / fwd_ms / 1e9,
                     "psa_fwd_frac_of_measured_peak": flops_fwd / fwd_ms / 1e9 / peaks["bf16_tflops"],
                     "psa_bwd_main_ms": bwd_ms, "psa_bwd_main_tflops": bwd_tflops,
-                    "psa_bwd_helpers_ms": att_ms - fwd_ms - bwd_ms,
+                    "psa_bwd_delta_clear_ms": kernel_ms["bwd_delta_clear"], "psa_bwd_convert_ms": kernel_ms["bwd_convert"],
+                    "timing": "CUDA events recorded by the library around each kernel, every pass of the timed region",
                     "dpo_logp_ms": klp_ms, "dpo_logp_gbs": logp_bytes / klp_ms / 1e6,
                     "dpo_logp_frac_of_hbm": {"measured": logp_bytes / klp_ms / 1e6 / peaks["hbm_gbs"],
                                              "nominal": logp_bytes / klp_ms / 1e6 / NOMINAL_HBM_GBS},
                     "dpo_logp_live_rows": live_rows, "dpo_logp_step_ms": lp_ms},
         "roofline": {"kernel": "psa_bwd_kernel<%d>" % d, "bound": "tensor", "achieved": bwd_tflops,
-                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": bwd_tflops / peaks["bf16_tflops"],
+                     "peak": peak_tc, "unit": "TFLOP/s", "frac": bwd_tflops / peak_tc,
+                     "frac_of_burst_peak": bwd_tflops / peaks["bf16_tflops"],
                      "scope": "this one kernel (the dominant one), not the attention forward + backward as a whole: "
                               "that is pct_of_bf16_peak",
-                     "peak_kind": "burst bf16 cuBLAS, of " + peaks["source"],
+                     "peak_kind": peak_kind,
                      "algorithmic_flops": flops_bwd, "algorithmic_bytes": T * (4 * Hq + 4 * Hkv) * d * 2,
                      "traffic": traffic, "traffic_source": traffic_note},
         "clocks": clk,

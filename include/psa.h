@@ -455,8 +455,9 @@ psa_status_t dpo_logp_bwd(const void* logits, int32_t logits_dtype, int64_t n_ro
  * pair of cudaEvent_t (passed as void*) that the next calls record on their stream
  * immediately before and after one chosen kernel, so that a benchmark can time that
  * kernel alone while it runs inside a whole step.
- *   which   0 = the psa_fwd kernel, 1 = the main psa_bwd kernel (without the
- *           delta / clear / convert helpers), 2 = the dpo_logp kernel
+ *   which   0 = the psa_fwd kernel, 1 = the main psa_bwd kernel (without its helpers),
+ *           2 = the dpo_logp kernel, 3 = psa_bwd's first helper (delta, and the clearing of
+ *           the dq accumulator), 4 = psa_bwd's last helper (dq accumulator -> bf16)
  *   start, stop   events created with timing enabled; pass NULL, NULL to unregister.
  * Process-global and not thread-safe; the events must outlive the calls they time.
  * Errors: INVALID_ARG (bad `which`, or only one of the two events given).

@@ -288,10 +288,12 @@ def dpo_logp(logits, targets, segment_ids, n_segments, fork_rows=None, fork_targ
     return out
 
 
-def psa_profile_events(which, start=None, stop=None):
+def psa_profile_events(which, start=None, stop=None, created=False):
     """Registers (or, with None, removes) a pair of torch.cuda.Event recorded right
-    before and after one kernel: 0 = psa_fwd, 1 = main psa_bwd kernel, 2 = dpo_logp."""
-    if start is not None:
+    before and after one kernel: 0 = psa_fwd, 1 = main psa_bwd kernel, 2 = dpo_logp,
+    3 = psa_bwd's delta / clear helper, 4 = psa_bwd's convert helper.  `created=True` says the
+    events have been recorded before (so their CUDA events exist) and skips the dummy record."""
+    if start is not None and not created:
         # torch creates the underlying cudaEvent lazily, on the first record
         start.record()
         stop.record()

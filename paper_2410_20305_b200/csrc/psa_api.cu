@@ -135,7 +135,8 @@ psa_status_t check_last_cuda_error(const char* where) {
   return PSA_ERR_CUDA;
 }
 
-ProfileEvents g_profile[3] = {{nullptr, nullptr}, {nullptr, nullptr}, {nullptr, nullptr}};
+ProfileEvents g_profile[5] = {{nullptr, nullptr}, {nullptr, nullptr}, {nullptr, nullptr}, {nullptr, nullptr},
+                              {nullptr, nullptr}};
 ProfileScope::ProfileScope(int which, void* s) : ev(g_profile[which]), stream(s) {
   if (ev.start) cudaEventRecord(cudaEvent_t(ev.start), cudaStream_t(stream));
 }
@@ -145,7 +146,7 @@ ProfileScope::~ProfileScope() {
 }  // namespace psa
 
 extern "C" psa_status_t psa_profile_events(int32_t which, void* start, void* stop) {
-  if (which < 0 || which > 2 || ((start == nullptr) != (stop == nullptr))) return PSA_ERR_INVALID_ARG;
+  if (which < 0 || which > 4 || ((start == nullptr) != (stop == nullptr))) return PSA_ERR_INVALID_ARG;
   psa::g_profile[which] = psa::ProfileEvents{start, stop};
   return PSA_OK;
 }

@@ -739,6 +739,7 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
 
   const int64_t n_rows = T * plan->Hq;
   {
+    ProfileScope prof(3, stream);
     const int64_t threads = n_rows * (D / 8);
     psa_bwd_delta_kernel<D><<<unsigned((threads + 255) / 256), 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(d_o), static_cast<const __nv_bfloat16*>(o), delta, dq_accum, n_rows, plan->T,
@@ -771,6 +772,7 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
     psa_bwd_kernel<D><<<grid, kBwdThreads, L::kRequest, stream>>>(tm_q, tm_k, tm_v, tm_do, tm_dq, tm_dk, tm_dv, prm);
   }
   if (!f32_out) {
+    ProfileScope prof(4, stream);
     const int64_t n_vec4 = n_rows * D / 4;
     psa_bwd_convert_kernel<<<unsigned((n_vec4 + 255) / 256), 256, 0, stream>>>(
         reinterpret_cast<const float4*>(dq_accum), static_cast<uint2*>(dq), n_vec4);

@@ -81,7 +81,7 @@ psa_status_t check_last_cuda_error(const char* where);
 
 // Optional event pairs recorded around one kernel (see psa_profile_events).
 struct ProfileEvents { void* start; void* stop; };
-extern ProfileEvents g_profile[3];
+extern ProfileEvents g_profile[5];
 struct ProfileScope {  // records start now and stop at scope exit, if registered
   ProfileEvents ev; void* stream;
   ProfileScope(int which, void* s);
