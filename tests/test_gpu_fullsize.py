@@ -106,6 +106,25 @@ def test_attention_on_the_bench_packs(workload):
                   % (workload, L, name, raw, raw32))
             assert raw_small <= TOL_O and excess <= TOL_O and raw32 <= TOL_O, (workload, name, raw, raw_small, excess, raw32)
 
+    # ---- (2b) the short-many pack is small enough for the dense oracle on every sample and ALL heads:
+    # every element of every output of the whole pack
+    if workload == 4:
+        worst = {}
+        for s in range(pack.n_samples):
+            lo, hi, sq, sk, sv, sdo = _sample_views(pack, s, (q, k, v, d_o), all_q, all_kv)
+            P, C, R = (int(x[s]) for x in (pack.prefix_len, pack.chosen_len, pack.rejected_len))
+            mask = orc.packed_mask([0, hi - lo], [P], [C], [R])
+            ro, rl = orc.attention_fwd(sq, sk, sv, mask)
+            rdq, rdk, rdv = orc.attention_bwd(sq, sk, sv, sdo, mask)
+            assert max_abs(o[lo:hi], ro) <= TOL_O and max_abs(lse[:, lo:hi], rl) <= TOL_LSE, (s, "whole pack")
+            for name, got, got32, ref in (("dq", dq[lo:hi], fq[lo:hi], rdq), ("dk", dk[lo:hi], fk[lo:hi], rdk),
+                                          ("dv", dv[lo:hi], fv[lo:hi], rdv)):
+                raw, raw_small, excess = grad_errors(got, ref)
+                raw32 = max_abs(got32, ref)
+                worst[name] = max(worst.get(name, 0.0), raw32)
+                assert raw_small <= TOL_O and excess <= TOL_O and raw32 <= TOL_O, (s, name, raw, raw_small, excess, raw32)
+        print("workload 4, whole pack, all heads, every element: worst raw error of the fp32 gradients", worst)
+
     # ---- (3) properties that hold at any size: finite everywhere, lse >= the row's own score
     assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
     assert all(torch.isfinite(t.float()).all() for t in (dq, dk, dv, fq, fk, fv))
