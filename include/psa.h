@@ -53,6 +53,8 @@ typedef enum {
 #define PSA_DEVSTAT_WAIT_EXPIRED 1 /* a bounded barrier wait gave up; outputs are invalid    */
 #define PSA_DEVSTAT_BAD_TARGET   2 /* dpo_logp: a scored target id was outside [0, vocab)    */
 #define PSA_DEVSTAT_BAD_SEGMENT  4 /* dpo_logp: a segment id was >= n_segments               */
+#define PSA_DEVSTAT_OUT_OF_BOUNDS 8 /* debug library only (libpsa_debug.so): a thread's own global
+                                       index fell outside its tensor; the access was skipped     */
 
 /* Flags of psa_plan(). */
 #define PSA_PLAN_HOST_ONLY 1 /* build the tile map on the host only; no CUDA call is made */
@@ -187,6 +189,19 @@ psa_status_t psa_bwd(const psa_plan_t* plan, const void* d_o, const void* q, con
                      const void* v, const void* o, const float* lse,
                      void* dq, void* dk, void* dv, void* workspace,
                      int32_t* device_status, void* stream);
+
+/*
+ * psa_selftest_bounds -- self test of the debug library's checked indices; the paper has no
+ * counterpart.  Tiles move by TMA, which clips every box to its tensor; the indices that threads
+ * form themselves (lse / delta words, ragged last tiles, fp32 gradient rows) are checked in
+ * libpsa_debug.so (the same sources built with -DPSA_DEBUG_BOUNDS): an index outside its tensor
+ * sets PSA_DEVSTAT_OUT_OF_BOUNDS and the access is skipped.  This call runs one index inside and
+ * one outside a 4-element tensor through that check: in the debug library *result = 1 and the bit
+ * is set; in the product library, where the check compiles to nothing, *result = 3 and no bit.
+ *   device_status, result   device int32 [1]
+ * Errors: INVALID_ARG, CUDA.
+ */
+psa_status_t psa_selftest_bounds(int32_t* device_status, int32_t* result, void* stream);
 
 /*
  * psa_bwd_f32 -- psa_bwd with fp32 gradient outputs (same computation, same kernels; the only

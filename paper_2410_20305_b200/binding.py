@@ -19,7 +19,7 @@ _lib = None
 PSA_PLAN_HOST_ONLY = 1
 PSA_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 PSA_DTYPE_F32, PSA_DTYPE_BF16 = 0, 1
-PSA_DEVSTAT_WAIT_EXPIRED, PSA_DEVSTAT_BAD_TARGET, PSA_DEVSTAT_BAD_SEGMENT = 1, 2, 4
+PSA_DEVSTAT_WAIT_EXPIRED, PSA_DEVSTAT_BAD_TARGET, PSA_DEVSTAT_BAD_SEGMENT, PSA_DEVSTAT_OUT_OF_BOUNDS = 1, 2, 4, 8
 
 EXPORTED_SYMBOLS = (
     "psa_status_string", "psa_plan", "psa_plan_upload", "psa_plan_destroy", "psa_plan_stats",
@@ -27,6 +27,7 @@ EXPORTED_SYMBOLS = (
     "psa_bwd_static_scratch", "dpo_loss", "dpo_logp_bwd", "psa_pack_ffd", "psa_position_ids", "psa_rope",
     "psa_step_host_arena_bytes", "psa_step_host", "simpo_loss", "orpo_loss", "psa_bwd_f32",
     "psa_check_device_status", "psa_selftest_wait_expiry", "psa_logp_labels", "psa_pack_ffd_emit",
+    "psa_selftest_bounds",
 )
 
 
@@ -38,19 +39,22 @@ class PsaError(RuntimeError):
 
 def load_library():
     """Loads libpsa.so (building it first if the sources are newer and nvcc is
-    present).  Raises if the library cannot be had."""
+    present).  Raises if the library cannot be had.  With PSA_DEBUG_LIB=1 in the environment the
+    debug library (libpsa_debug.so: the same code with checked global indices) is loaded instead."""
     global _lib
     if _lib is not None:
         return _lib
     from . import build as _build
+    debug = os.environ.get("PSA_DEBUG_LIB", "") not in ("", "0")
+    path = _build.LIB_DEBUG if debug else _LIB_PATH
     try:
-        _build.build()
+        _build.build(debug=debug)
     except Exception:
-        if not os.path.exists(_LIB_PATH):
+        if not os.path.exists(path):
             raise
-    if not os.path.exists(_LIB_PATH):
-        raise RuntimeError("libpsa.so is missing and could not be built: %s" % _LIB_PATH)
-    lib = C.CDLL(_LIB_PATH)
+    if not os.path.exists(path):
+        raise RuntimeError("%s is missing and could not be built" % path)
+    lib = C.CDLL(path)
     vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
     lib.psa_status_string.restype = C.c_char_p
     lib.psa_status_string.argtypes = [C.c_int]
@@ -67,6 +71,7 @@ def load_library():
     lib.psa_bwd_f32.argtypes = [vp] * 13
     lib.psa_check_device_status.argtypes = [i32]
     lib.psa_selftest_wait_expiry.argtypes = [vp, i64, vp, vp]
+    lib.psa_selftest_bounds.argtypes = [vp, vp, vp]
     lib.psa_logp_labels.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, C.POINTER(i32)]
     lib.psa_pack_ffd_emit.argtypes = [vp, vp, vp, i32, i32, i32, vp, C.POINTER(i32), vp, vp, vp, vp, vp, vp]
     lib.psa_profile_events.argtypes = [i32, vp, vp]
@@ -261,6 +266,12 @@ def psa_selftest_wait_expiry(status, limit_clocks, waited=None, stream=None):
     `waited` (int64 CUDA [1], optional) receives the clocks the wait lasted."""
     _check("psa_selftest_wait_expiry",
            load_library().psa_selftest_wait_expiry(_ptr(status), int(limit_clocks), _ptr(waited), _stream(stream)))
+
+
+def psa_selftest_bounds(status, result, stream=None):
+    """Runs one index inside and one outside a small tensor through the debug library's checked-index
+    macro (see psa.h); `status`, `result` are int32 CUDA [1]."""
+    _check("psa_selftest_bounds", load_library().psa_selftest_bounds(_ptr(status), _ptr(result), _stream(stream)))
 
 
 def dpo_logp(logits, targets, segment_ids, n_segments, fork_rows=None, fork_targets=None, fork_segments=None,

@@ -304,7 +304,7 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     auto load_stat = [&](int it) {
       const int64_t qrow = int64_t(rec.ds) + (entry_of(it) >> 2) * kTile + (wt & 127);
       float x = 0.f;
-      if (qrow < prm.T) {
+      if (qrow < prm.T && PSA_IN_BOUNDS(int64_t(head_of(it)) * prm.T + qrow, int64_t(prm.Hq) * prm.T, prm.status)) {
         const int64_t idx = int64_t(head_of(it)) * prm.T + qrow;
         x = wt < 128 ? prm.lse[idx] * kLog2e : prm.delta[idx];
       }
@@ -488,7 +488,8 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         for (int ch = 0; ch < DH / 32; ++ch) {
           uint32_t v[32];
           tmem_ld32_wait(tmem + lane_base + (which ? kColDK : kColDV) + half * DH + ch * 32, v);
-          if (kv_valid) {
+          if (kv_valid && PSA_IN_BOUNDS((row * prm.Hkv + hk) * D + half * DH + ch * 32 + 31, int64_t(prm.T) * prm.Hkv * D,
+                                        prm.status)) {
             float4* dst = reinterpret_cast<float4*>(dst_row + ch * 32);
 #pragma unroll
             for (int i = 0; i < 8; ++i)
@@ -546,7 +547,8 @@ psa_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       for (int ch = 0; ch < DH / 32; ++ch) {
         uint32_t v[32];
         tmem_ld32_wait(tmem + lane_base + (which ? kColDK : kColDV) + half * DH + ch * 32, v);
-        if (kv_valid) {
+        if (kv_valid && PSA_IN_BOUNDS((row * prm.Hkv + hk) * D + half * DH + ch * 32 + 31, int64_t(prm.T) * prm.Hkv * D,
+                                      prm.status)) {
           uint4* dst = reinterpret_cast<uint4*>(dst_row + ch * 32);
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -628,7 +630,7 @@ template <int D>
 __global__ void __launch_bounds__(256)
 psa_bwd_delta_kernel(const __nv_bfloat16* __restrict__ d_o, const __nv_bfloat16* __restrict__ o,
                      float* __restrict__ delta, float* __restrict__ dq_accum, int64_t n_rows /* T*Hq */, int32_t T,
-                     int32_t Hq) {
+                     int32_t Hq, int32_t* status) {
   constexpr int kLanes = D / 8;  // threads per (t, h) row
   const int64_t gid = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t row = gid / kLanes;
@@ -653,7 +655,7 @@ psa_bwd_delta_kernel(const __nv_bfloat16* __restrict__ d_o, const __nv_bfloat16*
   if (row < n_rows && part == 0) {
     const int64_t t = row / Hq;
     const int h = int(row % Hq);
-    delta[int64_t(h) * T + t] = acc;
+    if (PSA_IN_BOUNDS(int64_t(h) * T + t, int64_t(Hq) * T, status)) delta[int64_t(h) * T + t] = acc;
   }
 }
 
@@ -667,7 +669,8 @@ __global__ void __launch_bounds__(128)
 psa_bwd_delta_few_keys_kernel(const FewKeyRow* __restrict__ rows, const __nv_bfloat16* __restrict__ q,
                               const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
                               const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ lse,
-                              float* __restrict__ delta, int32_t T, int32_t Hq, int32_t Hkv, float scale_log2) {
+                              float* __restrict__ delta, int32_t T, int32_t Hq, int32_t Hkv, float scale_log2,
+                              int32_t* status) {
   const FewKeyRow rec = rows[blockIdx.x];
   const int h = blockIdx.y * 4 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -675,8 +678,8 @@ psa_bwd_delta_few_keys_kernel(const FewKeyRow* __restrict__ rows, const __nv_bfl
   const int hk = h / (Hq / Hkv);
   const int n_keys = rec.n_prompt + (rec.row - rec.rs_row + 1);   // < kFewKeys = 32
   float term = 0.f;
-  if (lane < n_keys) {
-    const int64_t key = lane < rec.n_prompt ? rec.ds + lane : rec.rs_row + (lane - rec.n_prompt);
+  const int64_t key = lane < rec.n_prompt ? rec.ds + lane : rec.rs_row + (lane - rec.n_prompt);
+  if (lane < n_keys && PSA_IN_BOUNDS(key, T, status) && PSA_IN_BOUNDS(rec.row, T, status)) {
     const uint4* q4 = reinterpret_cast<const uint4*>(q + (int64_t(rec.row) * Hq + h) * D);
     const uint4* g4 = reinterpret_cast<const uint4*>(d_o + (int64_t(rec.row) * Hq + h) * D);
     const uint4* k4 = reinterpret_cast<const uint4*>(k + (key * Hkv + hk) * D);
@@ -700,7 +703,7 @@ psa_bwd_delta_few_keys_kernel(const FewKeyRow* __restrict__ rows, const __nv_bfl
   }
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) term += __shfl_xor_sync(0xffffffffu, term, off);
-  if (lane == 0) delta[int64_t(h) * T + rec.row] = term;
+  if (lane == 0 && PSA_IN_BOUNDS(rec.row, T, status)) delta[int64_t(h) * T + rec.row] = term;
 }
 
 // dq = bf16(dq_accum).  Four independent 16-byte loads in flight per thread and streaming (evict-first)
@@ -754,13 +757,13 @@ psa_status_t launch_bwd_t(const psa_plan_t* plan, const void* d_o, const void* q
     const int64_t threads = n_rows * (D / 8);
     psa_bwd_delta_kernel<D><<<unsigned((threads + 255) / 256), 256, 0, stream>>>(
         static_cast<const __nv_bfloat16*>(d_o), static_cast<const __nv_bfloat16*>(o), delta, dq_accum, n_rows, plan->T,
-        plan->Hq);
+        plan->Hq, device_status);
   }
   if (!plan->few_key_rows.empty())
     psa_bwd_delta_few_keys_kernel<D><<<dim3(unsigned(plan->few_key_rows.size()), unsigned((plan->Hq + 3) / 4)), 128, 0, stream>>>(
         plan->d_few_key_rows, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
         static_cast<const __nv_bfloat16*>(v), static_cast<const __nv_bfloat16*>(d_o), lse, delta, plan->T, plan->Hq,
-        plan->Hkv, plan->scale * kLog2e);
+        plan->Hkv, plan->scale * kLog2e, device_status);
   BwdParams prm;
   prm.tiles = plan->d_kv_tiles;
   prm.entries = plan->d_bwd_entries;

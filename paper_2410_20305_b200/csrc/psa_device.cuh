@@ -74,6 +74,22 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const W
   }
 }
 
+// ---------------------------------------------------------------- debug build: checked global indices
+// Tiles move through TMA, whose tensor maps clip every box to the tensor.  The accesses that threads make
+// themselves (lse / delta words, ragged last tiles, fp32 gradient rows) go through PSA_IN_BOUNDS: in the debug
+// library (-DPSA_DEBUG_BOUNDS, libpsa_debug.so) an index outside [0, n) sets PSA_DEVSTAT_OUT_OF_BOUNDS in the
+// status word and the access is skipped; in the product library the macro is the constant true.
+#ifdef PSA_DEBUG_BOUNDS
+__device__ __forceinline__ bool index_in_bounds(long long i, long long n, int32_t* status) {
+  if (i >= 0 && i < n) return true;
+  if (status) atomicOr(status, PSA_DEVSTAT_OUT_OF_BOUNDS);
+  return false;
+}
+#define PSA_IN_BOUNDS(i, n, status) ::psa::dev::index_in_bounds((long long)(i), (long long)(n), (status))
+#else
+#define PSA_IN_BOUNDS(i, n, status) true
+#endif
+
 // ---------------------------------------------------------------- TMA
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

@@ -623,7 +623,8 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                        pack_bf16x2(__uint_as_float(v[8 * i + 4]) * inv_l, __uint_as_float(v[8 * i + 5]) * inv_l),
                        pack_bf16x2(__uint_as_float(v[8 * i + 6]) * inv_l, __uint_as_float(v[8 * i + 7]) * inv_l));
         }
-      } else if (row_valid) {
+      } else if (row_valid && PSA_IN_BOUNDS((row * prm.Hq + h) * D + hfz * (D / 2) + ch * 32 + 31,
+                                             int64_t(prm.T) * prm.Hq * D, prm.status)) {
         uint4* dst = reinterpret_cast<uint4*>(orow + ch * 32);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -636,7 +637,7 @@ psa_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
       }
     }
-    if (row_valid && hfz == 0) {
+    if (row_valid && hfz == 0 && PSA_IN_BOUNDS(int64_t(h) * prm.T + row, int64_t(prm.Hq) * prm.T, prm.status)) {
       const float mc = (m_run == -INFINITY) ? 0.f : m_run * c;
       prm.lse[int64_t(h) * prm.T + row] = (mc + log2f(l_run)) * 0.6931471805599453f;
     }

@@ -35,8 +35,22 @@ psa_wait_expiry_kernel(int32_t* status, long long limit_clocks, long long* waite
   if (threadIdx.x == 1) dev::mbar_wait(dev::smem_u32(&barrier_word), 0, ctx);
 }
 
+// One index inside and one outside a 4-element tensor through the checked-index macro.
+__global__ void psa_bounds_selftest_kernel(int32_t* status, int32_t* result) {
+  int32_t r = 0;
+  if (PSA_IN_BOUNDS(3, 4, status)) r |= 1;    // accepted in both libraries
+  if (PSA_IN_BOUNDS(4, 4, status)) r |= 2;    // accepted only where the macro is the constant true
+  *result = r;
+}
+
 }  // namespace
 }  // namespace psa
+
+extern "C" psa_status_t psa_selftest_bounds(int32_t* device_status, int32_t* result, void* stream) {
+  if (!device_status || !result) return PSA_ERR_INVALID_ARG;
+  psa::psa_bounds_selftest_kernel<<<1, 1, 0, cudaStream_t(stream)>>>(device_status, result);
+  return psa::check_last_cuda_error("psa_selftest_bounds launch");
+}
 
 extern "C" psa_status_t psa_selftest_wait_expiry(int32_t* device_status, int64_t limit_clocks, int64_t* spins_out,
                                                  void* stream) {
