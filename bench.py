@@ -13,8 +13,9 @@ same process and reported in the line's `workloads` object.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..4] [--impl reference]
 
-N > 1 (launched through torch.distributed.run) runs N independent replicas: the
-path has no exchange step, so there is no collective on the data path.
+N > 1 (launched through torch.distributed.run) shards the batch by packs: every rank
+takes a pack of its own (the packs of a batch are independent), so there is no
+collective on the data path; the report sums the ranks' work over the slowest time.
 """
 from __future__ import annotations
 
@@ -175,9 +176,29 @@ def max_over_ranks(values, device):
     return [float(x) for x in t.cpu()]
 
 
-def whole_job_tflops(flops_per_replica, world, ms):
-    """N independent replicas: the job's work is the sum, its time the slowest rank's."""
-    return world * flops_per_replica / ms / 1e9
+def sum_over_ranks(values, device):
+    """Element-wise sum of a list of floats over all ranks (identity on one rank): the work the
+    ranks did on their own packs.  Like max_over_ranks it reduces a few scalars of the report,
+    after the timed region; the data path has no collective."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t.cpu()]
+
+
+def whole_job_tflops(flops_all_ranks, ms):
+    """The packs of a batch are independent: every rank takes its own pack; the job's work is the
+    sum over the ranks, its time the slowest rank's."""
+    return flops_all_ranks / ms / 1e9
+
+
+def rank_pack(workload, rank):
+    """Rank 0 takes the configuration's own pack; every other rank draws another pack of the same
+    length distribution (pack sharding: one pack of the batch per GPU)."""
+    from paper_2410_20305_b200 import workloads as wl
+    return wl.config_pack(workload) if rank == 0 else wl.config_pack(workload, seed=1000 + workload + 7919 * rank)
 
 
 def oracle_sample_set(pack):
@@ -319,7 +340,7 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    pack = wl.config_pack(args.workload)
+    pack = rank_pack(args.workload, rank)
     if args.impl == "reference":
         return run_reference(args, pack, rank)
 
@@ -613,6 +634,7 @@ def main():
     # ---- max over ranks (replicas): whole-job value = sum of the replicas' useful flops / slowest time
     step_ms, att_ms, lp_ms, e2e_ms_max = max_over_ranks(
         [step_ms, att_ms, lp_ms, e2e["ms_per_step"] if e2e else 0.0], dev)
+    flops_all, tokens_all = sum_over_ranks([flops_fwd + flops_bwd, float(T)], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -620,7 +642,7 @@ def main():
 
     if all_rows:
         all_rows["frac_of_hbm"] = {"measured": all_rows["gbs"] / peaks["hbm_gbs"], "nominal": all_rows["gbs"] / NOMINAL_HBM_GBS}
-    value = whole_job_tflops(flops_fwd + flops_bwd, world, att_ms)
+    value = whole_job_tflops(flops_all, att_ms)
     att_min_bytes = T * (6 * Hq + 6 * Hkv) * d * 2
     bwd_ms, fwd_ms, klp_ms = kernel_ms["bwd"], kernel_ms["fwd"], kernel_ms["logp"]
     # A region of half a second or more runs under the power cap at a reduced SM clock: the peak to
@@ -644,7 +666,8 @@ def main():
                    "n_q_heads": Hq, "n_kv_heads": Hkv, "head_dim": d, "useful_pairs_per_head": U,
                    "live_tiles": plan0.live_tiles, "partial_tiles": plan0.partial_tiles, "logits": [T, VOCAB],
                    "l2": "inputs larger than L2 (q, o, dO, dq are %.0f MB each; logits %.1f GB)" % (T * Hq * d * 2 / 1e6, T * VOCAB * 2 / 1e9),
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+                   "parallelism": ("one pack per GPU (%d packs, %d tokens in all; rank 0's pack is described here), "
+                                   "no collective on the data path" % (world, int(tokens_all))) if world > 1 else "single GPU"},
         "inner_repeats": inner,
         "timed_region": {"passes": n_pass, "ms": timed_ms,
                          "note": "each of the --steps steps is run inner_repeats times so that the region lasts at least "
@@ -674,8 +697,8 @@ def main():
         "attention_min_hbm": {"bytes": att_min_bytes, "gbs": att_min_bytes / att_ms / 1e6,
                               "frac_of_hbm": {"measured": att_min_bytes / att_ms / 1e6 / peaks["hbm_gbs"],
                                               "nominal": att_min_bytes / att_ms / 1e6 / NOMINAL_HBM_GBS}},
-        "tokens_per_s": world * T / (step_ms * 1e-3),
-        "attention_tokens_per_s": world * T / (att_ms * 1e-3),
+        "tokens_per_s": tokens_all / (step_ms * 1e-3),
+        "attention_tokens_per_s": tokens_all / (att_ms * 1e-3),
         "kernels": {"psa_fwd_ms": fwd_ms, "psa_fwd_tflops": flops_fwd / fwd_ms / 1e9,
                     "psa_fwd_frac_of_measured_peak": flops_fwd / fwd_ms / 1e9 / peaks["bf16_tflops"],
                     "psa_bwd_main_ms": bwd_ms, "psa_bwd_main_tflops": bwd_tflops,
@@ -704,7 +727,7 @@ def main():
         "paper_context": "paper reports 1.1-1.5x (1.3-1.6x with packing) end-to-end training speedups on 8xH100; context, not the target",
     }
     if e2e:
-        e2e["value"] = whole_job_tflops(flops_fwd + flops_bwd, world, e2e_ms_max)
+        e2e["value"] = whole_job_tflops(flops_all, e2e_ms_max)
         e2e["ms_per_step"] = e2e_ms_max
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:

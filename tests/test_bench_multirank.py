@@ -1,5 +1,6 @@
-"""The N > 1 path of bench.py on CPU: two gloo ranks, replicas only.  The only collective
-is the max-reduction of the ranks' timings; the reference arm prints on rank 0 alone."""
+"""The N > 1 path of bench.py on CPU: two gloo ranks, one pack per rank.  The only collectives
+are the max-reduction of the ranks' timings and the sum of their work, after the timed region;
+the reference arm prints on rank 0 alone."""
 import json
 import os
 import subprocess
@@ -18,6 +19,8 @@ def _worker(rank, world, port, out):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
     dist.init_process_group("gloo", rank=rank, world_size=world)
     got = bench.max_over_ranks([1.0 + rank, 5.0 - rank, 2.0], "cpu")
+    pack = bench.rank_pack(1, rank)
+    got += bench.sum_over_ranks([10.0 + rank, float(pack.total_tokens)], "cpu")
     dist.barrier()
     dist.destroy_process_group()
     out.put((rank, got))
@@ -34,15 +37,25 @@ def test_max_over_ranks_two_gloo_ranks():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    assert results[0] == results[1] == [2.0, 5.0, 2.0]
-
-
-def test_whole_job_value_is_sum_of_replicas_over_slowest_time():
     sys.path.insert(0, ROOT)
     import bench
-    assert bench.whole_job_tflops(2e12, 1, 1.0) == 2000.0
-    assert bench.whole_job_tflops(2e12, 8, 2.0) == 8000.0
+    packs = [bench.rank_pack(1, r) for r in range(2)]
+    assert packs[0].total_tokens != packs[1].total_tokens or list(packs[0].prefix_len) != list(packs[1].prefix_len)
+    assert results[0] == results[1] == [2.0, 5.0, 2.0, 21.0, float(packs[0].total_tokens + packs[1].total_tokens)]
+
+
+def test_whole_job_value_is_sum_of_the_ranks_work_over_slowest_time():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.whole_job_tflops(2e12, 1.0) == 2000.0
+    assert bench.whole_job_tflops(16e12, 2.0) == 8000.0
     assert bench.max_over_ranks([3.0], "cpu") == [3.0]       # single process: identity
+    assert bench.sum_over_ranks([3.0, 4.0], "cpu") == [3.0, 4.0]
+    # rank 0 keeps the configuration's own pack; the others draw from the same length distribution
+    from paper_2410_20305_b200 import workloads as wl
+    assert list(bench.rank_pack(3, 0).cu_seqlens) == list(wl.config_pack(3).cu_seqlens)
+    other = bench.rank_pack(3, 5)
+    assert other.pack_len == 32768 and 0.85 * 32768 <= other.total_tokens <= 32768
 
 
 def test_reference_arm_prints_one_line_on_rank_zero_only():
