@@ -19,7 +19,7 @@ def test_library_exports_every_declared_symbol():
     lib = B.load_library()
     header = open(os.path.join(ROOT, "include", "psa.h")).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(psa_[a-z_]+|dpo_lo[a-z_]*|simpo_[a-z_]+|orpo_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(psa_[a-z0-9_]+|dpo_lo[a-z0-9_]*|simpo_[a-z_]+|orpo_[a-z_]+)\s*\(", header))
     declared.discard("psa_status_t")
     assert declared, "no declarations found"
     assert set(B.EXPORTED_SYMBOLS) >= declared
