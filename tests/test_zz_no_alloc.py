@@ -69,7 +69,9 @@ def test_the_call_allocates_no_device_memory():
     for _ in range(3):
         B.psa_bwd_static_scratch(plan, d_o, q, k, v, o, lse, *got)
     torch.cuda.synchronize()
-    assert torch.cuda.mem_get_info()[0] == free0, "device free memory changed across the calls"
+    # (an allocation by the calls would lower the device's free memory; memory freed meanwhile by someone
+    # else sharing the GPU may raise it)
+    assert torch.cuda.mem_get_info()[0] >= free0, "device free memory dropped across the calls"
     assert {key: torch.cuda.memory_stats().get(key, 0) for key in keys} == stats0
 
 
