@@ -101,3 +101,31 @@ def test_run_twice_outputs_are_identical_where_the_order_of_additions_is_fixed()
         assert torch.equal(a, b)
     assert (runs[0][6] - runs[1][6]).abs().max().item() <= 1e-5        # fp32 dq: order of the adds only
     assert (runs[0][7].float() - runs[1][7].float()).abs().max().item() <= 2.0 ** -6   # bf16 dq: at most one rounding step
+
+
+def test_two_streams_two_packs_do_not_disturb_each_other():
+    """Forward and backward of two different packs enqueued on two streams at the same time, each with its own
+    plan, outputs and workspace: the library keeps no hidden state between calls, so each result must be
+    bit-identical (o, lse, dk, dv) to the same pack run alone."""
+    packs = [wl.random_pack(201, 4, 500, 8, 2, 128), wl.random_pack(202, 5, 400, 4, 4, 64)]
+    ins = [[t.cuda() for t in wl.attention_inputs(p, 60 + i)] for i, p in enumerate(packs)]
+    plans = [device_plan(p) for p in packs]
+    alone = []
+    for plan, (q, k, v, d_o) in zip(plans, ins):
+        o, lse = B.psa_fwd(plan, q, k, v)
+        alone.append((o, lse) + B.psa_bwd(plan, d_o, q, k, v, o, lse))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    both = [None, None]
+    for rep in range(3):
+        for i in (0, 1):
+            q, k, v, d_o = ins[i]
+            s = streams[i].cuda_stream
+            with torch.cuda.stream(streams[i]):
+                o, lse = B.psa_fwd(plans[i], q, k, v, stream=s)
+                both[i] = (o, lse) + B.psa_bwd(plans[i], d_o, q, k, v, o, lse, stream=s)
+    torch.cuda.synchronize()
+    for i in (0, 1):
+        for a, b in zip(alone[i][:2] + alone[i][3:], both[i][:2] + both[i][3:]):
+            assert torch.equal(a, b)
+        assert (alone[i][2].float() - both[i][2].float()).abs().max().item() <= 2.0 ** -6     # dq: order of the adds
